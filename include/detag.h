@@ -1,0 +1,160 @@
+/*
+ * detag.h - C ABI of the B200 (sm_100a) DeTAG step library.
+ *
+ * DeTAG = decentralized stochastic gradient tracking with by-phase accelerated gossip
+ * (arXiv 2006.08085, Algorithms 2 and 3).  The library applies one DeTAG iteration at once
+ * to all n simulated workers, each holding a flat float32 parameter vector of length d, on
+ * one GPU.
+ *
+ * Conventions used by every entry point
+ *   - Return value: DETAG_OK (0) or a negative DETAG_ERR_* code.  Nothing throws, traps or
+ *     exits; detag_last_error() gives a text for the last failure on a state.
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA global memory of
+ *     the device that is current when the call is made.  The library allocates no device
+ *     memory: the caller owns every device buffer (state arrays and the workspace) and
+ *     keeps it alive and unaliased while it is bound.  detag_destroy frees host memory only.
+ *   - `stream` is a CUDA stream handle (cudaStream_t / CUstream) passed as void*; NULL is
+ *     the legacy default stream.  Calls documented "asynchronous" only enqueue work.
+ *   - State arrays are row-major [n][ld] float32: worker i's vector starts at element
+ *     i*ld; ld >= d, ld a multiple of 4, base addresses 16-byte aligned.
+ *   - A state is used by one host thread at a time.
+ *
+ * One step, in the order the kernels execute it (Algorithm 2; gradient evaluated at the new
+ * model, folded into the tracker before the next gossip):
+ *     y~  = AG_K(y)                      Algorithm 3 on the tracker
+ *     x~  = AG_K(x)                      Algorithm 3 on the model
+ *     x'  = x~ - alpha * y~              model update of Algorithm 2
+ *     g'  = a o (x' - c) + sigma * xi    stochastic gradient of f_i(x) = 1/2 sum_j a_ij (x_j - c_ij)^2
+ *     y'  = y~ + g' - g                  tracker update of Algorithm 2 (with the stored float32 g')
+ * so the `y` buffer always holds the tracker with the newest gradient already folded in,
+ * and each of x, y, g, a, c is read once and x, y, g written once per step.
+ */
+#ifndef DETAG_H
+#define DETAG_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct detag_state detag_state; /* opaque, lives in host memory */
+
+enum {
+  DETAG_OK = 0,
+  DETAG_ERR_ARG = -1,            /* null pointer, non-positive size, misaligned or too small buffer */
+  DETAG_ERR_CSR = -2,            /* row_ptr not monotone, column out of range, unsorted or duplicate */
+  DETAG_ERR_NOT_STOCHASTIC = -3, /* some row or column sum differs from 1 by more than 1e-9 */
+  DETAG_ERR_NOT_SYMMETRIC = -4,  /* eta had to be derived but the matrix is not symmetric */
+  DETAG_ERR_UNSUPPORTED = -5,    /* n or nnz beyond what the kernels' shared-memory plan holds */
+  DETAG_ERR_UNBOUND = -6,        /* a call that needs buffers came before detag_bind */
+  DETAG_ERR_CUDA = -7,           /* a CUDA runtime call or launch failed (text in detag_last_error) */
+  DETAG_ERR_TIMEOUT = -8,        /* a bounded device-side wait gave up (reported by detag_status) */
+  DETAG_ERR_SPECTRUM = -9        /* lambda >= 1: disconnected or bipartite graph, no valid eta */
+};
+
+/* Kernel variants of the gossip part of the step; all compute the same result. */
+enum {
+  DETAG_VARIANT_AUTO = 0,  /* host cost model picks */
+  DETAG_VARIANT_CSR = 1,   /* K rounds of neighbour-indexed sums over the CSR rows, slab staged on chip */
+  DETAG_VARIANT_DENSE = 2, /* one product with the host-precomputed polynomial P_K(M), n <= 64 */
+  DETAG_VARIANT_RING = 3   /* K rounds with register-blocked halo exchange, circulant ring matrices only */
+};
+
+/*
+ * Spectrum of a symmetric gossip matrix and the accelerated-gossip momentum.
+ * Paper: Section "Protocol Layer" (lambda = max(|lambda_2|, |lambda_n|)) and Algorithm 3
+ * (eta = (1 - sqrt(1 - lambda^2)) / (1 + sqrt(1 - lambda^2))).
+ * Host only.  The matrix is n x n in CSR (host pointers: row_ptr[n+1], col_idx[nnz], vals[nnz]).
+ * Any output pointer may be NULL.  Errors: ARG, CSR, NOT_SYMMETRIC, UNSUPPORTED (n > 2048),
+ * SPECTRUM (lambda >= 1; the eigenvalue outputs are still written).
+ */
+int detag_spectral(int n, const int32_t* row_ptr, const int32_t* col_idx, const double* vals,
+                   double* lambda2, double* lambda_min, double* lambda, double* eta);
+
+/*
+ * Create a state for n workers with d coordinates each.
+ * The CSR arrays (host; copied) describe the matrix M that a gossip round applies row-wise,
+ * z'_i = sum_j M[i][j] z_j, i.e. M[i][j] is the paper's W_ji (Eq. "gossip update",
+ * Algorithm 3).  Columns sorted and unique within a row; M doubly stochastic.
+ * K >= 1 is the number of accelerated-gossip rounds per step (the paper's phase length R),
+ * alpha the step size of Algorithm 2, eta the momentum of Algorithm 3; pass NaN to have it
+ * derived from the spectrum (needs a symmetric M).  Host only; no device work.
+ * Errors: ARG, CSR, NOT_STOCHASTIC, NOT_SYMMETRIC, SPECTRUM, UNSUPPORTED (n > 1024).
+ */
+int detag_create(detag_state** out, int n, int64_t d, const int32_t* row_ptr, const int32_t* col_idx,
+                 const double* vals, int K, double eta, double alpha);
+
+/* Bytes of device workspace detag_bind needs for this state (graph tables, polynomial, partial sums). */
+int detag_workspace_bytes(const detag_state* s, size_t* bytes);
+
+/*
+ * Bind the caller's device buffers (see the layout conventions above):
+ *   x, y, g : state, read and written by detag_init / detag_step
+ *   a, c    : objective data, read only
+ *   workspace: at least detag_workspace_bytes() bytes, 256-byte aligned; the call fills it with
+ *              the graph tables (synchronous copies on the current device).
+ * Rebinding is allowed (e.g. to step another coordinate shard with the same graph).
+ * Errors: ARG, CUDA.
+ */
+int detag_bind(detag_state* s, int64_t ld, float* x, float* y, float* g, const float* a, const float* c,
+               void* workspace, size_t workspace_bytes);
+
+/*
+ * Optional observer: when y_gossip (device, [n][ld] float32) is non-NULL, every later step also
+ * stores the tracker right after its gossip (y~ above, the value Algorithm 2 uses in the model
+ * update).  NULL (the default) switches it off.  Costs one extra array write per step.
+ */
+int detag_observe_gossiped_tracker(detag_state* s, float* y_gossip);
+
+/*
+ * Noise of the stochastic gradient oracle (Section "Setting", oracle class): xi is standard
+ * normal, a pure function of (seed, step, worker, global coordinate); sigma = 0 gives the exact
+ * gradient.  coord_offset is the global index of column 0 of the bound arrays (for coordinate
+ * shards).  Defaults: sigma 0, seed 0, offset 0.
+ */
+int detag_set_noise(detag_state* s, double sigma, uint64_t seed, int64_t coord_offset);
+
+/* Force a kernel variant (DETAG_VARIANT_*).  Errors: ARG, UNSUPPORTED (variant not applicable to this M). */
+int detag_set_variant(detag_state* s, int variant);
+/* The variant the next detag_step will run (never AUTO). */
+int detag_get_variant(const detag_state* s, int* variant);
+
+/*
+ * Initial state of Algorithm 2 as the task fixes it: g = stochastic gradient at the bound x
+ * (noise of step 0), y = g.  Sets the step counter to 0.  Asynchronous.  Errors: UNBOUND, CUDA.
+ */
+int detag_init(detag_state* s, void* stream);
+
+/*
+ * One DeTAG iteration for all workers (Algorithm 2 with Algorithm 3 as the gossip; see the
+ * step listing at the top).  Asynchronous; the step counter advances by one at enqueue time.
+ * Errors: UNBOUND, CUDA (launch failure).  Device-side problems surface in detag_status.
+ */
+int detag_step(detag_state* s, void* stream);
+
+/*
+ * Consensus error of the model, ||X - Xbar 1^T||_F^2 = sum_j sum_i (x_ij - mean_i x_ij)^2
+ * (the quantity bounded in the proof of Theorem 3), accumulated in float64 in a fixed order.
+ * Enqueues on `stream`, waits for it, writes *host_out.  Errors: ARG, UNBOUND, CUDA.
+ */
+int detag_consensus_error(detag_state* s, void* stream, double* host_out);
+
+/* Step counter t (number of completed steps; enters the noise counter).  set_step is for resume. */
+int detag_get_step(const detag_state* s, int64_t* t);
+int detag_set_step(detag_state* s, int64_t t);
+
+/* Waits for `stream`, then returns the device status word: DETAG_OK or DETAG_ERR_TIMEOUT. */
+int detag_status(detag_state* s, void* stream);
+
+/* Text of the last error on this state ("" if none).  Owned by the state. */
+const char* detag_last_error(const detag_state* s);
+
+/* Frees the host-side state.  Device buffers stay the caller's. */
+int detag_destroy(detag_state* s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DETAG_H */

@@ -1,0 +1,101 @@
+// Internal declarations shared by the host API and the kernel launchers of libdetag.
+#ifndef DETAG_INTERNAL_H
+#define DETAG_INTERNAL_H
+
+#include <cstddef>
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "detag.h"
+
+typedef struct CUstream_st* cudaStream_t;
+
+namespace detag {
+
+constexpr int kMaxWorkers = 1024;       // detag_create limit on n
+constexpr int kMaxDenseWorkers = 64;    // dense-polynomial variant limit on n
+constexpr int kMaxPartials = 2048;      // per-CTA partial sums of the consensus-error reduction
+constexpr size_t kWsAlign = 256;
+
+// Everything a step / init / reduction kernel needs, passed by value.
+struct StepParams {
+  int n;
+  int nnz;
+  int K;
+  int S;           // slab width in coordinates (power of two)
+  int log2S;
+  long long d;
+  long long ld;
+  long long num_slabs;
+  long long coord_offset;  // global index of column 0 (noise counter)
+  float* x;
+  float* y;
+  float* g;
+  const float* a;
+  const float* c;
+  float* y_obs;  // optional gossiped-tracker output, may be null
+  const int32_t* row_ptr;
+  const int32_t* col_idx;
+  const double* vals;
+  const double* poly;  // dense P_K(M), row-major n x n (null when n > kMaxDenseWorkers)
+  double eta;
+  double alpha;
+  double sigma;
+  uint32_t seed_lo, seed_hi;
+  uint32_t t_noise;  // step index that enters the noise counter
+  int* status;
+};
+
+// host helpers (spectral.cpp)
+int validate_csr(int n, const int32_t* row_ptr, const int32_t* col_idx, const double* vals);
+void csr_to_dense(int n, const int32_t* row_ptr, const int32_t* col_idx, const double* vals, std::vector<double>& m);
+bool is_symmetric(int n, const std::vector<double>& m, double tol);
+void jacobi_eigenvalues(int n, std::vector<double>& a, std::vector<double>& ev);
+double eta_from_lambda(double lam);
+
+// kernel launchers; each returns a cudaError_t value as int (0 = success)
+int launch_init_gradient(const StepParams& p, int sm_count, cudaStream_t stream);
+int plan_step_csr(StepParams& p, int smem_optin_bytes);  // chooses S; DETAG_ERR_UNSUPPORTED if nothing fits
+int launch_step_csr(const StepParams& p, int sm_count, cudaStream_t stream);
+int launch_consensus_error(const StepParams& p, double* partials, double* result, int sm_count, cudaStream_t stream);
+
+}  // namespace detag
+
+struct detag_state {
+  int n = 0;
+  long long d = 0;
+  int K = 0;
+  double eta = 0.0, alpha = 0.0;
+  std::vector<int32_t> row_ptr, col_idx;
+  std::vector<double> vals;
+  std::vector<double> poly;  // P_K(M) when n <= kMaxDenseWorkers
+  int variant_forced = DETAG_VARIANT_AUTO;
+
+  bool bound = false;
+  long long ld = 0;
+  float *x = nullptr, *y = nullptr, *g = nullptr;
+  const float *a = nullptr, *c = nullptr;
+  float* y_obs = nullptr;
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  int* d_status = nullptr;
+  double* d_result = nullptr;
+  int32_t* d_row_ptr = nullptr;
+  int32_t* d_col_idx = nullptr;
+  double* d_vals = nullptr;
+  double* d_poly = nullptr;
+  double* d_partials = nullptr;
+
+  double sigma = 0.0;
+  uint64_t seed = 0;
+  long long coord_offset = 0;
+  long long t = 0;
+
+  int device = -1;
+  int sm_count = 0;
+  int smem_optin = 0;
+  std::string err;
+};
+
+#endif  // DETAG_INTERNAL_H
