@@ -1,0 +1,119 @@
+// Stand-alone kernels around the step: the stochastic gradient of the synthetic objective
+// (used for the initial state) and the consensus-error reduction.
+#include <cuda_runtime.h>
+
+#include "detag_internal.h"
+#include "noise.cuh"
+
+namespace detag {
+
+namespace {
+
+constexpr int kAuxThreads = 256;
+
+// g = a (x - c) + sigma xi_t and y = g: the initial state y_0 = g(x_0) of the tracker.
+// One thread handles the four workers 4q..4q+3 of one coordinate (one Philox call).
+__global__ void __launch_bounds__(kAuxThreads) init_gradient_kernel(const StepParams p) {
+  const int nq = (p.n + 3) >> 2;
+  const long long items = static_cast<long long>(nq) * p.d;
+  const double sigma = p.sigma;
+  for (long long it = blockIdx.x * static_cast<long long>(kAuxThreads) + threadIdx.x; it < items;
+       it += static_cast<long long>(gridDim.x) * kAuxThreads) {
+    const int q = static_cast<int>(it / p.d);
+    const long long j = it - static_cast<long long>(q) * p.d;
+    float xi[4] = {0.f, 0.f, 0.f, 0.f};
+    if (sigma != 0.0)
+      normal_quad(p.seed_lo, p.seed_hi, static_cast<unsigned long long>(p.coord_offset + j), q, p.t_noise, xi);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const int i = 4 * q + w;
+      if (i < p.n) {
+        const long long off = static_cast<long long>(i) * p.ld + j;
+        const double g = fma(static_cast<double>(p.a[off]),
+                             static_cast<double>(p.x[off]) - static_cast<double>(p.c[off]),
+                             sigma * static_cast<double>(xi[w]));
+        const float gf = static_cast<float>(g);
+        p.g[off] = gf;
+        p.y[off] = gf;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Per coordinate: mean over workers, then the sum of squared deviations (two passes, float64).
+// Per CTA: warp-shuffle tree, then a fixed-order sum over the warps -> partials[blockIdx.x].
+__global__ void __launch_bounds__(kAuxThreads) consensus_partial_kernel(const StepParams p, double* partials) {
+  __shared__ double warp_part[kAuxThreads / 32];
+  double acc = 0.0;
+  const double inv_n = 1.0 / static_cast<double>(p.n);
+  for (long long j = blockIdx.x * static_cast<long long>(kAuxThreads) + threadIdx.x; j < p.d;
+       j += static_cast<long long>(gridDim.x) * kAuxThreads) {
+    double sum = 0.0;
+    for (int i = 0; i < p.n; ++i) sum += static_cast<double>(p.x[static_cast<long long>(i) * p.ld + j]);
+    const double mean = sum * inv_n;
+    double ss = 0.0;
+    for (int i = 0; i < p.n; ++i) {
+      const double dev = static_cast<double>(p.x[static_cast<long long>(i) * p.ld + j]) - mean;
+      ss = fma(dev, dev, ss);
+    }
+    acc += ss;
+  }
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int w = 0; w < kAuxThreads / 32; ++w) s += warp_part[w];
+    partials[blockIdx.x] = s;
+  }
+}
+
+// Single CTA: fixed-order sum of the partials.
+__global__ void __launch_bounds__(kAuxThreads) consensus_final_kernel(const double* partials, int count,
+                                                                      double* result) {
+  __shared__ double warp_part[kAuxThreads / 32];
+  double acc = 0.0;
+  for (int k = threadIdx.x; k < count; k += kAuxThreads) acc += partials[k];
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int w = 0; w < kAuxThreads / 32; ++w) s += warp_part[w];
+    *result = s;
+  }
+}
+
+}  // namespace
+
+int launch_init_gradient(const StepParams& p, int sm_count, cudaStream_t stream) {
+  const long long items = static_cast<long long>((p.n + 3) / 4) * p.d;
+  if (items <= 0) return 0;
+  long long grid = (items + kAuxThreads - 1) / kAuxThreads;
+  const long long cap = static_cast<long long>(sm_count) * 16;
+  if (grid > cap) grid = cap;
+  init_gradient_kernel<<<static_cast<unsigned>(grid), kAuxThreads, 0, stream>>>(p);
+  return static_cast<int>(cudaGetLastError());
+}
+
+int launch_consensus_error(const StepParams& p, double* partials, double* result, int sm_count,
+                           cudaStream_t stream) {
+  long long grid = (p.d + kAuxThreads - 1) / kAuxThreads;
+  long long cap = static_cast<long long>(sm_count) * 8;
+  if (cap > kMaxPartials) cap = kMaxPartials;
+  if (grid > cap) grid = cap;
+  if (grid < 1) grid = 1;
+  consensus_partial_kernel<<<static_cast<unsigned>(grid), kAuxThreads, 0, stream>>>(p, partials);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return static_cast<int>(e);
+  consensus_final_kernel<<<1, kAuxThreads, 0, stream>>>(partials, static_cast<int>(grid), result);
+  return static_cast<int>(cudaGetLastError());
+}
+
+}  // namespace detag
