@@ -1,0 +1,331 @@
+// Host side of the C ABI declared in include/detag.h: argument checking, the host-side numerics
+// (momentum, polynomial of the gossip matrix), workspace layout and kernel launches.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "detag_internal.h"
+
+using detag::StepParams;
+
+namespace {
+
+size_t align_up(size_t v) { return (v + detag::kWsAlign - 1) / detag::kWsAlign * detag::kWsAlign; }
+
+struct WsLayout {
+  size_t status, result, row_ptr, col_idx, vals, poly, partials, total;
+};
+
+WsLayout ws_layout(const detag_state* s) {
+  WsLayout l{};
+  size_t off = 0;
+  l.status = off;
+  l.result = off + 64;
+  off += detag::kWsAlign;
+  l.row_ptr = off;
+  off += align_up((s->n + 1) * sizeof(int32_t));
+  l.col_idx = off;
+  off += align_up(s->col_idx.size() * sizeof(int32_t));
+  l.vals = off;
+  off += align_up(s->vals.size() * sizeof(double));
+  l.poly = off;
+  off += align_up(s->poly.size() * sizeof(double));
+  l.partials = off;
+  off += align_up(detag::kMaxPartials * sizeof(double));
+  l.total = off;
+  return l;
+}
+
+int fail(detag_state* s, int code, const char* what) {
+  if (s) s->err = what;
+  return code;
+}
+
+int fail_cuda(detag_state* s, int cuda_code, const char* where) {
+  if (s) {
+    char buf[256];
+    std::snprintf(buf, sizeof buf, "%s: %s", where, cudaGetErrorString(static_cast<cudaError_t>(cuda_code)));
+    s->err = buf;
+  }
+  return DETAG_ERR_CUDA;
+}
+
+// P_K(M) by the matrix form of Algorithm 3: P_{-1} = P_0 = I, P_{r+1} = (1+eta) M P_r - eta P_{r-1}.
+void gossip_polynomial(const detag_state* s, std::vector<double>& out) {
+  const int n = s->n;
+  std::vector<double> prev(static_cast<size_t>(n) * n, 0.0), cur, next(static_cast<size_t>(n) * n);
+  for (int i = 0; i < n; ++i) prev[static_cast<size_t>(i) * n + i] = 1.0;
+  cur = prev;
+  for (int r = 0; r < s->K; ++r) {
+    for (int i = 0; i < n; ++i) {
+      for (int j = 0; j < n; ++j) {
+        double acc = 0.0;
+        for (int k = s->row_ptr[i]; k < s->row_ptr[i + 1]; ++k)
+          acc += s->vals[k] * cur[static_cast<size_t>(s->col_idx[k]) * n + j];
+        next[static_cast<size_t>(i) * n + j] = (1.0 + s->eta) * acc - s->eta * prev[static_cast<size_t>(i) * n + j];
+      }
+    }
+    prev.swap(cur);
+    cur.swap(next);
+  }
+  out = cur;
+}
+
+StepParams make_params(const detag_state* s) {
+  StepParams p{};
+  p.n = s->n;
+  p.nnz = static_cast<int>(s->col_idx.size());
+  p.K = s->K;
+  p.d = s->d;
+  p.ld = s->ld;
+  p.coord_offset = s->coord_offset;
+  p.x = s->x;
+  p.y = s->y;
+  p.g = s->g;
+  p.a = s->a;
+  p.c = s->c;
+  p.y_obs = s->y_obs;
+  p.row_ptr = s->d_row_ptr;
+  p.col_idx = s->d_col_idx;
+  p.vals = s->d_vals;
+  p.poly = s->d_poly;
+  p.eta = s->eta;
+  p.alpha = s->alpha;
+  p.sigma = s->sigma;
+  p.seed_lo = static_cast<uint32_t>(s->seed & 0xffffffffu);
+  p.seed_hi = static_cast<uint32_t>(s->seed >> 32);
+  p.status = s->d_status;
+  return p;
+}
+
+int resolve_variant(const detag_state* s) {
+  if (s->variant_forced != DETAG_VARIANT_AUTO) return s->variant_forced;
+  return DETAG_VARIANT_CSR;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+int detag_create(detag_state** out, int n, int64_t d, const int32_t* row_ptr, const int32_t* col_idx,
+                 const double* vals, int K, double eta, double alpha) {
+  if (!out) return DETAG_ERR_ARG;
+  *out = nullptr;
+  if (n <= 0 || d <= 0 || K < 1 || !std::isfinite(alpha)) return DETAG_ERR_ARG;
+  int rc = detag::validate_csr(n, row_ptr, col_idx, vals);
+  if (rc != DETAG_OK) return rc;
+  if (n > detag::kMaxWorkers) return DETAG_ERR_UNSUPPORTED;
+  const int nnz = row_ptr[n];
+  // doubly stochastic: every row and column sums to one
+  std::vector<double> col_sum(n, 0.0);
+  for (int i = 0; i < n; ++i) {
+    double row_sum = 0.0;
+    for (int k = row_ptr[i]; k < row_ptr[i + 1]; ++k) {
+      row_sum += vals[k];
+      col_sum[col_idx[k]] += vals[k];
+    }
+    if (std::fabs(row_sum - 1.0) > 1e-9) return DETAG_ERR_NOT_STOCHASTIC;
+  }
+  for (int j = 0; j < n; ++j)
+    if (std::fabs(col_sum[j] - 1.0) > 1e-9) return DETAG_ERR_NOT_STOCHASTIC;
+
+  if (std::isnan(eta)) {
+    double lam = 0.0;
+    rc = detag_spectral(n, row_ptr, col_idx, vals, nullptr, nullptr, &lam, &eta);
+    if (rc != DETAG_OK) return rc;
+  } else if (!std::isfinite(eta)) {
+    return DETAG_ERR_ARG;
+  }
+
+  detag_state* s = new (std::nothrow) detag_state();
+  if (!s) return DETAG_ERR_ARG;
+  s->n = n;
+  s->d = d;
+  s->K = K;
+  s->eta = eta;
+  s->alpha = alpha;
+  s->row_ptr.assign(row_ptr, row_ptr + n + 1);
+  s->col_idx.assign(col_idx, col_idx + nnz);
+  s->vals.assign(vals, vals + nnz);
+  if (n <= detag::kMaxDenseWorkers) gossip_polynomial(s, s->poly);
+  *out = s;
+  return DETAG_OK;
+}
+
+int detag_workspace_bytes(const detag_state* s, size_t* bytes) {
+  if (!s || !bytes) return DETAG_ERR_ARG;
+  *bytes = ws_layout(s).total;
+  return DETAG_OK;
+}
+
+int detag_bind(detag_state* s, int64_t ld, float* x, float* y, float* g, const float* a, const float* c,
+               void* workspace, size_t workspace_bytes) {
+  if (!s) return DETAG_ERR_ARG;
+  if (!x || !y || !g || !a || !c || !workspace) return fail(s, DETAG_ERR_ARG, "detag_bind: null buffer");
+  if (ld < s->d || (ld & 3) != 0) return fail(s, DETAG_ERR_ARG, "detag_bind: ld must be >= d and a multiple of 4");
+  if (!aligned16(x) || !aligned16(y) || !aligned16(g) || !aligned16(a) || !aligned16(c))
+    return fail(s, DETAG_ERR_ARG, "detag_bind: state arrays must be 16-byte aligned");
+  if ((reinterpret_cast<uintptr_t>(workspace) % detag::kWsAlign) != 0)
+    return fail(s, DETAG_ERR_ARG, "detag_bind: workspace must be 256-byte aligned");
+  const WsLayout l = ws_layout(s);
+  if (workspace_bytes < l.total) return fail(s, DETAG_ERR_ARG, "detag_bind: workspace too small");
+
+  cudaError_t e = cudaGetDevice(&s->device);
+  if (e != cudaSuccess) return fail_cuda(s, e, "cudaGetDevice");
+  e = cudaDeviceGetAttribute(&s->sm_count, cudaDevAttrMultiProcessorCount, s->device);
+  if (e != cudaSuccess) return fail_cuda(s, e, "cudaDeviceGetAttribute(sm count)");
+  e = cudaDeviceGetAttribute(&s->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, s->device);
+  if (e != cudaSuccess) return fail_cuda(s, e, "cudaDeviceGetAttribute(shared memory)");
+
+  unsigned char* base = static_cast<unsigned char*>(workspace);
+  s->d_status = reinterpret_cast<int*>(base + l.status);
+  s->d_result = reinterpret_cast<double*>(base + l.result);
+  s->d_row_ptr = reinterpret_cast<int32_t*>(base + l.row_ptr);
+  s->d_col_idx = reinterpret_cast<int32_t*>(base + l.col_idx);
+  s->d_vals = reinterpret_cast<double*>(base + l.vals);
+  s->d_poly = s->poly.empty() ? nullptr : reinterpret_cast<double*>(base + l.poly);
+  s->d_partials = reinterpret_cast<double*>(base + l.partials);
+
+  e = cudaMemset(base, 0, detag::kWsAlign);
+  if (e == cudaSuccess)
+    e = cudaMemcpy(s->d_row_ptr, s->row_ptr.data(), s->row_ptr.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess)
+    e = cudaMemcpy(s->d_col_idx, s->col_idx.data(), s->col_idx.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess)
+    e = cudaMemcpy(s->d_vals, s->vals.data(), s->vals.size() * sizeof(double), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess && s->d_poly)
+    e = cudaMemcpy(s->d_poly, s->poly.data(), s->poly.size() * sizeof(double), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return fail_cuda(s, e, "detag_bind: workspace upload");
+
+  s->ld = ld;
+  s->x = x;
+  s->y = y;
+  s->g = g;
+  s->a = a;
+  s->c = c;
+  s->ws = workspace;
+  s->ws_bytes = workspace_bytes;
+  s->bound = true;
+  return DETAG_OK;
+}
+
+int detag_observe_gossiped_tracker(detag_state* s, float* y_gossip) {
+  if (!s) return DETAG_ERR_ARG;
+  if (y_gossip && !aligned16(y_gossip)) return fail(s, DETAG_ERR_ARG, "observer buffer must be 16-byte aligned");
+  s->y_obs = y_gossip;
+  return DETAG_OK;
+}
+
+int detag_set_noise(detag_state* s, double sigma, uint64_t seed, int64_t coord_offset) {
+  if (!s) return DETAG_ERR_ARG;
+  if (!std::isfinite(sigma) || sigma < 0.0 || coord_offset < 0)
+    return fail(s, DETAG_ERR_ARG, "detag_set_noise: bad value");
+  s->sigma = sigma;
+  s->seed = seed;
+  s->coord_offset = coord_offset;
+  return DETAG_OK;
+}
+
+int detag_set_variant(detag_state* s, int variant) {
+  if (!s) return DETAG_ERR_ARG;
+  switch (variant) {
+    case DETAG_VARIANT_AUTO:
+    case DETAG_VARIANT_CSR:
+      break;
+    case DETAG_VARIANT_DENSE:
+    case DETAG_VARIANT_RING:
+      return fail(s, DETAG_ERR_UNSUPPORTED, "detag_set_variant: variant not available for this matrix");
+    default:
+      return fail(s, DETAG_ERR_ARG, "detag_set_variant: unknown variant");
+  }
+  s->variant_forced = variant;
+  return DETAG_OK;
+}
+
+int detag_get_variant(const detag_state* s, int* variant) {
+  if (!s || !variant) return DETAG_ERR_ARG;
+  *variant = resolve_variant(s);
+  return DETAG_OK;
+}
+
+int detag_init(detag_state* s, void* stream) {
+  if (!s) return DETAG_ERR_ARG;
+  if (!s->bound) return fail(s, DETAG_ERR_UNBOUND, "detag_init before detag_bind");
+  StepParams p = make_params(s);
+  p.t_noise = 0;
+  const int e = detag::launch_init_gradient(p, s->sm_count, static_cast<cudaStream_t>(stream));
+  if (e != 0) return fail_cuda(s, e, "detag_init launch");
+  s->t = 0;
+  return DETAG_OK;
+}
+
+int detag_step(detag_state* s, void* stream) {
+  if (!s) return DETAG_ERR_ARG;
+  if (!s->bound) return fail(s, DETAG_ERR_UNBOUND, "detag_step before detag_bind");
+  StepParams p = make_params(s);
+  p.t_noise = static_cast<uint32_t>(s->t + 1);
+  int e = 0;
+  switch (resolve_variant(s)) {
+    case DETAG_VARIANT_CSR:
+    default: {
+      const int rc = detag::plan_step_csr(p, s->smem_optin);
+      if (rc != DETAG_OK) return fail(s, rc, "detag_step: graph too large for the shared-memory plan");
+      e = detag::launch_step_csr(p, s->sm_count, static_cast<cudaStream_t>(stream));
+    }
+  }
+  if (e != 0) return fail_cuda(s, e, "detag_step launch");
+  s->t += 1;
+  return DETAG_OK;
+}
+
+int detag_consensus_error(detag_state* s, void* stream, double* host_out) {
+  if (!s || !host_out) return DETAG_ERR_ARG;
+  if (!s->bound) return fail(s, DETAG_ERR_UNBOUND, "detag_consensus_error before detag_bind");
+  const StepParams p = make_params(s);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int e = detag::launch_consensus_error(p, s->d_partials, s->d_result, s->sm_count, st);
+  if (e != 0) return fail_cuda(s, e, "detag_consensus_error launch");
+  cudaError_t ce = cudaMemcpyAsync(host_out, s->d_result, sizeof(double), cudaMemcpyDeviceToHost, st);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+  if (ce != cudaSuccess) return fail_cuda(s, ce, "detag_consensus_error copy");
+  return DETAG_OK;
+}
+
+int detag_get_step(const detag_state* s, int64_t* t) {
+  if (!s || !t) return DETAG_ERR_ARG;
+  *t = s->t;
+  return DETAG_OK;
+}
+
+int detag_set_step(detag_state* s, int64_t t) {
+  if (!s || t < 0) return DETAG_ERR_ARG;
+  s->t = t;
+  return DETAG_OK;
+}
+
+int detag_status(detag_state* s, void* stream) {
+  if (!s) return DETAG_ERR_ARG;
+  if (!s->bound) return fail(s, DETAG_ERR_UNBOUND, "detag_status before detag_bind");
+  int word = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(&word, s->d_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail_cuda(s, e, "detag_status");
+  if (word != 0) return fail(s, DETAG_ERR_TIMEOUT, "a device-side wait gave up");
+  return DETAG_OK;
+}
+
+const char* detag_last_error(const detag_state* s) { return s ? s->err.c_str() : ""; }
+
+int detag_destroy(detag_state* s) {
+  if (!s) return DETAG_ERR_ARG;
+  delete s;
+  return DETAG_OK;
+}
+
+}  // extern "C"
