@@ -1,0 +1,222 @@
+"""GPU-vs-oracle parity through the C ABI (needs a B200).
+
+Bars (floating point): after one step max |err| <= 1e-5 (1 + |ref|) per element; over a trajectory the
+relative L2 error of every state array is <= 1e-4 at every step.  The folded tracker the library stores
+telescopes against the *stored float32* gradient, so its per-element bound carries that value's
+half-ulp, 2^-24 |g'|, on top.
+"""
+import numpy as np
+import pytest
+
+from oracle import detag_oracle as orc
+from paper_2006_08085_b200 import binding as B
+from paper_2006_08085_b200 import build, inputs
+from paper_2006_08085_b200.session import Session
+from parity import HALF_ULP32, one_step_from_rounded_state, oracle_problem, rel_l2, worst_ratio
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+
+
+def _variants_for(m, K):
+    """Every kernel variant that accepts this matrix (CSR always does)."""
+    out = [B.DETAG_VARIANT_CSR]
+    st = B.detag_create(m.n, 8, m.row_ptr, m.col_idx, m.vals, K, 0.1, 0.1)
+    try:
+        for v in (B.DETAG_VARIANT_DENSE, B.DETAG_VARIANT_RING):
+            try:
+                B.detag_set_variant(st, v)
+                out.append(v)
+            except B.DetagError:
+                pass
+    finally:
+        B.detag_destroy(st)
+    return out
+
+
+def _random_objective(rng, n, d, scale=1.0):
+    a = rng.uniform(0.5, 2.0, (n, d)).astype(np.float32)
+    c = (scale * (rng.standard_normal((n, d)) + np.arange(n)[:, None] - n / 2)).astype(np.float32)
+    return a, c
+
+
+def _check_one_step(m, K, eta, alpha, a, c, x0, sigma, seed, j0=0, variants=None):
+    """One step from the oracle's float32-rounded initial state; every observable per element."""
+    n, d = a.shape
+    p = oracle_problem(m, K, eta, alpha, a, c, sigma, seed, j0)
+    (x32, y32, g32), (x_ref, yg_ref, g_ref, yf_ref) = one_step_from_rounded_state(p, x0)
+    worst = {}
+    for v in variants or _variants_for(m, K):
+        with Session(m, d, K, eta, alpha, a, c, x32, sigma, seed, coord_offset=j0, observe_gossip=True,
+                     variant=v) as s:
+            s.upload("y", y32)
+            s.upload("g", g32)
+            B.detag_set_step(s.state, 0)
+            s.step()
+            s.status()
+            r = {
+                "x": worst_ratio(s.download("x"), x_ref),
+                "y_gossip": worst_ratio(s.download("y_gossip"), yg_ref),
+                "g": worst_ratio(s.download("g"), g_ref),
+                "y": worst_ratio(s.download("y"), yf_ref, extra=HALF_ULP32 * np.abs(g_ref)),
+            }
+        assert max(r.values()) <= 1.0, (v, r)
+        worst[v] = r
+    return worst
+
+
+def _check_trajectory(m, K, eta, alpha, a, c, x0, sigma, seed, steps, j0=0, variants=None, bound=1e-4):
+    """Whole pipeline on the GPU (init + steps) against the pure float64 oracle run, every step."""
+    n, d = a.shape
+    p = oracle_problem(m, K, eta, alpha, a, c, sigma, seed, j0)
+    ref = []
+    orc.run(p, x0, steps, observe=lambda s: ref.append((s.x.copy(), orc.folded_tracker(s), s.g_new.copy())))
+    for v in variants or _variants_for(m, K):
+        with Session(m, d, K, eta, alpha, a, c, x0, sigma, seed, coord_offset=j0, variant=v) as s:
+            s.init()
+            for t in range(steps + 1):
+                if t > 0:
+                    s.step()
+                errs = {k: rel_l2(s.download(k), r) for k, r in zip(("x", "y", "g"), ref[t])}
+                if t == 0:
+                    errs.pop("x")  # x0 is an input (and may be all zero)
+                assert max(errs.values()) <= bound, (v, t, errs)
+            s.status()
+            ce = s.consensus_error()
+            assert ce == pytest.approx(orc.consensus_error(ref[-1][0]), rel=1e-4, abs=1e-12)
+
+
+# ----------------------------------------------------------------------------- small and edge cases
+@pytest.mark.parametrize("n,d,K", [(3, 1, 1), (5, 37, 2), (8, 300, 3), (8, 129, 16), (7, 4, 5), (12, 1025, 4)])
+def test_small_rings_ragged_sizes(n, d, K):
+    rng = np.random.default_rng(n * 1000 + d)
+    m = inputs.metropolis_weights(inputs.ring_graph(n))
+    eta = orc.spectrum(m.to_dense()).eta
+    a, c = _random_objective(rng, n, d)
+    x0 = rng.standard_normal((n, d)).astype(np.float32)
+    _check_one_step(m, K, eta, 0.05, a, c, x0, 0.1, 11)
+    _check_trajectory(m, K, eta, 0.05, a, c, x0, 0.1, 11, steps=6)
+
+
+def test_irregular_graph_and_noise_free():
+    rng = np.random.default_rng(5)
+    m = inputs.metropolis_weights(inputs.path_graph(9))  # degrees 1 and 2
+    eta = orc.spectrum(m.to_dense()).eta
+    a, c = _random_objective(rng, 9, 77)
+    x0 = np.zeros((9, 77), dtype=np.float32)
+    _check_one_step(m, 3, eta, 0.05, a, c, x0, 0.0, 0)
+    _check_trajectory(m, 3, eta, 0.05, a, c, x0, 0.0, 0, steps=8)
+
+
+def test_non_symmetric_matrix_is_applied_row_wise():
+    rng = np.random.default_rng(6)
+    m = inputs.directed_cycle_blend(6, 0.45, 0.35)
+    a, c = _random_objective(rng, 6, 50)
+    x0 = rng.standard_normal((6, 50)).astype(np.float32)
+    _check_one_step(m, 4, 0.3, 0.05, a, c, x0, 0.1, 3)
+
+
+def test_average_consensus_and_dsgt_special_cases():
+    rng = np.random.default_rng(7)
+    a, c = _random_objective(rng, 6, 40)
+    x0 = rng.standard_normal((6, 40)).astype(np.float32)
+    _check_one_step(inputs.average_consensus_matrix(6), 1, 0.0, 0.1, a, c, x0, 0.1, 1)
+    _check_one_step(inputs.metropolis_weights(inputs.ring_graph(6)), 1, 0.0, 0.1, a, c, x0, 0.1, 1)  # DSGT
+
+
+def test_coordinate_offset_enters_the_noise_counter():
+    rng = np.random.default_rng(8)
+    m = inputs.metropolis_weights(inputs.ring_graph(8))
+    a, c = _random_objective(rng, 8, 64)
+    x0 = np.zeros((8, 64), dtype=np.float32)
+    _check_one_step(m, 2, 0.25, 0.05, a, c, x0, 0.1, 9, j0=(1 << 32) + 12345, variants=[B.DETAG_VARIANT_CSR])
+
+
+def test_padded_leading_dimension_is_left_untouched():
+    rng = np.random.default_rng(9)
+    m = inputs.metropolis_weights(inputs.ring_graph(5))
+    a, c = _random_objective(rng, 5, 30)
+    for v in _variants_for(m, 2):
+        with Session(m, 30, 2, 0.2, 0.05, a, c, np.zeros((5, 30), np.float32), 0.1, 1, ld=48, variant=v) as s:
+            for t in (s.x, s.y, s.g):
+                t[:, 30:] = 777.0
+            s.init()
+            s.step(3)
+            s.status()
+            for t in (s.x, s.y, s.g):
+                assert bool((t[:, 30:] == 777.0).all())
+
+
+def test_large_worker_count_n_256_and_n_1000():
+    rng = np.random.default_rng(10)
+    for n, d, K in ((256, 70, 3), (1000, 9, 2)):
+        m = inputs.metropolis_weights(inputs.ring_graph(n))
+        a, c = _random_objective(rng, n, d, scale=0.05)
+        x0 = np.zeros((n, d), dtype=np.float32)
+        _check_one_step(m, K, 0.4, 0.01, a, c, x0, 0.1, 2)
+
+
+def test_misuse_is_reported_not_faulted():
+    import torch
+
+    m = inputs.metropolis_weights(inputs.ring_graph(4))
+    st = B.detag_create(4, 16, m.row_ptr, m.col_idx, m.vals, 2, 0.1, 0.1)
+    try:
+        buf = torch.zeros(4 * 16 + 64, dtype=torch.float32, device="cuda:0")
+        ws = torch.zeros(B.detag_workspace_bytes(st) + 256, dtype=torch.uint8, device="cuda:0")
+        wsp = ws.data_ptr() + (-ws.data_ptr()) % 256
+        good = buf.data_ptr()
+        for args in ((15, good, good, good, good, good, wsp, ws.numel() - 256),  # ld < d
+                     (18, good, good, good, good, good, wsp, ws.numel() - 256),  # ld not a multiple of 4
+                     (16, good + 4, good, good, good, good, wsp, ws.numel() - 256),  # misaligned
+                     (16, good, good, good, good, good, wsp + 8, ws.numel() - 256),  # workspace misaligned
+                     (16, good, good, good, good, good, wsp, 64)):  # workspace too small
+            with pytest.raises(B.DetagError) as e:
+                B.detag_bind(st, *args)
+            assert e.value.code == B.DETAG_ERR_ARG
+        with pytest.raises(B.DetagError) as e:
+            B.detag_consensus_error(st)
+        assert e.value.code == B.DETAG_ERR_UNBOUND
+    finally:
+        B.detag_destroy(st)
+
+
+# ----------------------------------------------------------------------------- the five configurations
+def _config_case(name, d):
+    cfg = inputs.CONFIGS[name]
+    cfg = cfg.with_d(min(d, cfg.d))
+    m = inputs.gossip_matrix(cfg)
+    eta = orc.spectrum(m.to_dense()).eta
+    a, c, x0 = inputs.objective_data(cfg)
+    return cfg, m, eta, a, c, x0
+
+
+@pytest.mark.parametrize("name,d", [("cfg1", 4096), ("cfg2", 270_000), ("cfg3", 20_003), ("cfg4", 5_001),
+                                    ("cfg5", 40_001)])
+def test_config_one_step_per_element(name, d):
+    cfg, m, eta, a, c, x0 = _config_case(name, d)
+    _check_one_step(m, cfg.K, eta, cfg.alpha, a, c, x0, cfg.sigma, cfg.seed)
+
+
+@pytest.mark.parametrize("name,d,steps", [("cfg1", 4096, 100), ("cfg2", 30_001, 100), ("cfg3", 3_001, 100),
+                                          ("cfg4", 601, 50), ("cfg5", 6_001, 100)])
+def test_config_trajectory(name, d, steps):
+    cfg, m, eta, a, c, x0 = _config_case(name, d)
+    _check_trajectory(m, cfg.K, eta, cfg.alpha, a, c, x0, cfg.sigma, cfg.seed, steps=steps)
+
+
+def test_consensus_error_matches_definition():
+    rng = np.random.default_rng(12)
+    m = inputs.metropolis_weights(inputs.ring_graph(16))
+    x = (rng.standard_normal((16, 100_003)) * 3 + 50).astype(np.float32)
+    a = np.ones_like(x)
+    with Session(m, x.shape[1], 2, 0.1, 0.1, a, a, x) as s:
+        assert s.consensus_error() == pytest.approx(orc.consensus_error(x), rel=1e-12)
+        assert s.consensus_error() == s.consensus_error()  # fixed summation order
+    cons = np.tile(rng.standard_normal((1, 1000)).astype(np.float32), (16, 1))
+    with Session(m, 1000, 2, 0.1, 0.1, a[:, :1000], a[:, :1000], cons) as s:
+        assert s.consensus_error() == 0.0

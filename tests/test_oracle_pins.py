@@ -319,3 +319,22 @@ def test_consensus_error_definition():
     x = np.array([[1.0, 2.0], [3.0, 2.0], [5.0, 2.0]])
     assert orc.consensus_error(x) == pytest.approx(8.0)
     assert orc.consensus_error(np.tile(np.arange(4.0), (5, 1))) == 0.0
+
+
+def test_parity_helper_is_the_same_cycle_cut_elsewhere():
+    """The storage convention used on the GPU side (gossip, gradient, then fold) is the oracle's step
+    (fold, gossip, gradient) cut at another point: on float32-exact data both give identical numbers."""
+    from parity import one_step_from_rounded_state
+
+    rng = np.random.default_rng(0)
+    w = inputs.metropolis_weights(inputs.ring_graph(6))
+    a = rng.choice([0.5, 1.0, 2.0], (6, 9)).astype(np.float32)
+    c = rng.integers(-4, 5, (6, 9)).astype(np.float32)
+    x0 = rng.integers(-3, 4, (6, 9)).astype(np.float32)
+    p = _problem(w, 3, 0.25, 0.0625, a, c, 0.0)
+    (x32, y32, g32), (x1, yg1, g1, yf1) = one_step_from_rounded_state(p, x0)
+    s0 = orc.init_state(p, x0)
+    assert np.array_equal(x32, s0.x) and np.array_equal(g32, s0.g_new)  # nothing was lost in the rounding
+    s1 = orc.step(p, s0)
+    assert np.array_equal(s1.x, x1) and np.array_equal(s1.y, yg1) and np.array_equal(s1.g_new, g1)
+    assert np.array_equal(orc.folded_tracker(s1), yf1)
