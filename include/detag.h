@@ -141,6 +141,23 @@ int detag_step(detag_state* s, void* stream);
  */
 int detag_consensus_error(detag_state* s, void* stream, double* host_out);
 
+/*
+ * One DeTAG iteration (same arithmetic as detag_step) on state that lives in HOST memory: x, y, g
+ * (read and written) and a, c (read) are host arrays [n][ld_host] float32, page-locked if the
+ * copies are to overlap.  The coordinate axis is cut into chunks; each chunk is copied to the
+ * device, stepped and copied back, two chunks in flight on two internal streams (the step never
+ * mixes coordinates, so chunks are independent).  `staging` is caller-owned device memory of
+ * `staging_bytes` >= detag_host_staging_bytes(s, chunk_coords): it holds the graph tables and two
+ * chunk slots; buffers bound with detag_bind are not touched and need not exist.
+ * Ordering: the work starts after everything enqueued on `stream` so far and `stream` waits for
+ * it; the call itself returns without waiting.  The step counter advances by one.
+ * Errors: ARG (null/misaligned pointers, staging too small for a 128-coordinate chunk), CUDA.
+ */
+int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* g, const float* a, const float* c,
+                    void* staging, size_t staging_bytes, void* stream);
+/* Device bytes detag_step_host needs to run with chunks of `chunk_coords` coordinates (a multiple of 128). */
+int detag_host_staging_bytes(const detag_state* s, int64_t chunk_coords, size_t* bytes);
+
 /* Step counter t (number of completed steps; enters the noise counter).  set_step is for resume. */
 int detag_get_step(const detag_state* s, int64_t* t);
 int detag_set_step(detag_state* s, int64_t t);

@@ -54,6 +54,8 @@ SIGNATURES = {
     "detag_get_variant": (ctypes.c_int, [_P, ctypes.POINTER(ctypes.c_int)]),
     "detag_init": (ctypes.c_int, [_P, _P]),
     "detag_step": (ctypes.c_int, [_P, _P]),
+    "detag_step_host": (ctypes.c_int, [_P, ctypes.c_int64, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P]),
+    "detag_host_staging_bytes": (ctypes.c_int, [_P, ctypes.c_int64, ctypes.POINTER(ctypes.c_size_t)]),
     "detag_consensus_error": (ctypes.c_int, [_P, _P, _F64P]),
     "detag_get_step": (ctypes.c_int, [_P, ctypes.POINTER(ctypes.c_int64)]),
     "detag_set_step": (ctypes.c_int, [_P, ctypes.c_int64]),
@@ -172,6 +174,20 @@ def detag_init(state, stream=None) -> None:
 
 def detag_step(state, stream=None) -> None:
     _check(lib().detag_step(state, _stream_handle(stream)), "detag_step", state)
+
+
+def detag_step_host(state, ld_host: int, x, y, g, a, c, staging, staging_bytes: int, stream=None) -> None:
+    """x, y, g, a, c: host tensors (page-locked for overlap) or raw host addresses; staging: device memory."""
+    _check(lib().detag_step_host(state, ld_host, _dev_ptr(x), _dev_ptr(y), _dev_ptr(g), _dev_ptr(a), _dev_ptr(c),
+                                 _dev_ptr(staging), int(staging_bytes), _stream_handle(stream)),
+           "detag_step_host", state)
+
+
+def detag_host_staging_bytes(state, chunk_coords: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().detag_host_staging_bytes(state, int(chunk_coords), ctypes.byref(out)), "detag_host_staging_bytes",
+           state)
+    return int(out.value)
 
 
 def detag_consensus_error(state, stream=None) -> float:

@@ -108,6 +108,31 @@ int resolve_variant(const detag_state* s) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+int query_device(detag_state* s) {
+  cudaError_t e = cudaGetDevice(&s->device);
+  if (e != cudaSuccess) return fail_cuda(s, e, "cudaGetDevice");
+  e = cudaDeviceGetAttribute(&s->sm_count, cudaDevAttrMultiProcessorCount, s->device);
+  if (e != cudaSuccess) return fail_cuda(s, e, "cudaDeviceGetAttribute(sm count)");
+  e = cudaDeviceGetAttribute(&s->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, s->device);
+  if (e != cudaSuccess) return fail_cuda(s, e, "cudaDeviceGetAttribute(shared memory)");
+  return DETAG_OK;
+}
+
+// Picks the kernel variant, plans it for the sizes in `p` and launches it.
+int launch_step(detag_state* s, StepParams& p, cudaStream_t stream) {
+  int e = 0;
+  switch (resolve_variant(s)) {
+    case DETAG_VARIANT_CSR:
+    default: {
+      const int rc = detag::plan_step_csr(p, s->smem_optin);
+      if (rc != DETAG_OK) return fail(s, rc, "graph too large for the shared-memory plan");
+      e = detag::launch_step_csr(p, s->sm_count, stream);
+    }
+  }
+  if (e != 0) return fail_cuda(s, e, "step kernel launch");
+  return DETAG_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -175,12 +200,9 @@ int detag_bind(detag_state* s, int64_t ld, float* x, float* y, float* g, const f
   const WsLayout l = ws_layout(s);
   if (workspace_bytes < l.total) return fail(s, DETAG_ERR_ARG, "detag_bind: workspace too small");
 
-  cudaError_t e = cudaGetDevice(&s->device);
-  if (e != cudaSuccess) return fail_cuda(s, e, "cudaGetDevice");
-  e = cudaDeviceGetAttribute(&s->sm_count, cudaDevAttrMultiProcessorCount, s->device);
-  if (e != cudaSuccess) return fail_cuda(s, e, "cudaDeviceGetAttribute(sm count)");
-  e = cudaDeviceGetAttribute(&s->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, s->device);
-  if (e != cudaSuccess) return fail_cuda(s, e, "cudaDeviceGetAttribute(shared memory)");
+  const int qrc = query_device(s);
+  if (qrc != DETAG_OK) return qrc;
+  cudaError_t e = cudaSuccess;
 
   unsigned char* base = static_cast<unsigned char*>(workspace);
   s->d_status = reinterpret_cast<int*>(base + l.status);
@@ -269,16 +291,101 @@ int detag_step(detag_state* s, void* stream) {
   if (!s->bound) return fail(s, DETAG_ERR_UNBOUND, "detag_step before detag_bind");
   StepParams p = make_params(s);
   p.t_noise = static_cast<uint32_t>(s->t + 1);
-  int e = 0;
-  switch (resolve_variant(s)) {
-    case DETAG_VARIANT_CSR:
-    default: {
-      const int rc = detag::plan_step_csr(p, s->smem_optin);
-      if (rc != DETAG_OK) return fail(s, rc, "detag_step: graph too large for the shared-memory plan");
-      e = detag::launch_step_csr(p, s->sm_count, static_cast<cudaStream_t>(stream));
-    }
+  const int rc = launch_step(s, p, static_cast<cudaStream_t>(stream));
+  if (rc != DETAG_OK) return rc;
+  s->t += 1;
+  return DETAG_OK;
+}
+
+int detag_host_staging_bytes(const detag_state* s, int64_t chunk_coords, size_t* bytes) {
+  if (!s || !bytes || chunk_coords < 128 || (chunk_coords % 128) != 0) return DETAG_ERR_ARG;
+  *bytes = ws_layout(s).total + static_cast<size_t>(2) * 5 * s->n * static_cast<size_t>(chunk_coords) * sizeof(float);
+  return DETAG_OK;
+}
+
+int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* g, const float* a, const float* c,
+                    void* staging, size_t staging_bytes, void* stream) {
+  if (!s) return DETAG_ERR_ARG;
+  if (!x || !y || !g || !a || !c || !staging) return fail(s, DETAG_ERR_ARG, "detag_step_host: null buffer");
+  if (ld_host < s->d) return fail(s, DETAG_ERR_ARG, "detag_step_host: ld_host < d");
+  if ((reinterpret_cast<uintptr_t>(staging) % detag::kWsAlign) != 0)
+    return fail(s, DETAG_ERR_ARG, "detag_step_host: staging must be 256-byte aligned");
+  const WsLayout l = ws_layout(s);
+  const size_t per_coord = static_cast<size_t>(2) * 5 * s->n * sizeof(float);
+  if (staging_bytes < l.total + per_coord * 128)
+    return fail(s, DETAG_ERR_ARG, "detag_step_host: staging too small for a 128-coordinate chunk");
+  long long chunk = static_cast<long long>((staging_bytes - l.total) / per_coord) / 128 * 128;
+  const long long d_up = (s->d + 127) / 128 * 128;
+  if (chunk > d_up) chunk = d_up;
+
+  int rc = query_device(s);
+  if (rc != DETAG_OK) return rc;
+  cudaError_t e = cudaSuccess;
+  for (int k = 0; k < 2 && e == cudaSuccess; ++k)
+    if (!s->host_stream[k]) e = cudaStreamCreateWithFlags(&s->host_stream[k], cudaStreamNonBlocking);
+  for (int k = 0; k < 3 && e == cudaSuccess; ++k)
+    if (!s->host_event[k]) e = cudaEventCreateWithFlags(&s->host_event[k], cudaEventDisableTiming);
+  if (e != cudaSuccess) return fail_cuda(s, e, "detag_step_host: stream/event creation");
+
+  cudaStream_t user = static_cast<cudaStream_t>(stream);
+  unsigned char* base = static_cast<unsigned char*>(staging);
+  // graph tables at the head of the staging area, ordered on the caller's stream
+  e = cudaMemsetAsync(base, 0, detag::kWsAlign, user);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(base + l.row_ptr, s->row_ptr.data(), s->row_ptr.size() * sizeof(int32_t),
+                        cudaMemcpyHostToDevice, user);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(base + l.col_idx, s->col_idx.data(), s->col_idx.size() * sizeof(int32_t),
+                        cudaMemcpyHostToDevice, user);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(base + l.vals, s->vals.data(), s->vals.size() * sizeof(double), cudaMemcpyHostToDevice, user);
+  if (e == cudaSuccess && !s->poly.empty())
+    e = cudaMemcpyAsync(base + l.poly, s->poly.data(), s->poly.size() * sizeof(double), cudaMemcpyHostToDevice, user);
+  if (e == cudaSuccess) e = cudaEventRecord(s->host_event[2], user);
+  for (int k = 0; k < 2 && e == cudaSuccess; ++k) e = cudaStreamWaitEvent(s->host_stream[k], s->host_event[2], 0);
+  if (e != cudaSuccess) return fail_cuda(s, e, "detag_step_host: table upload");
+
+  StepParams p = make_params(s);
+  p.row_ptr = reinterpret_cast<int32_t*>(base + l.row_ptr);
+  p.col_idx = reinterpret_cast<int32_t*>(base + l.col_idx);
+  p.vals = reinterpret_cast<double*>(base + l.vals);
+  p.poly = s->poly.empty() ? nullptr : reinterpret_cast<double*>(base + l.poly);
+  p.status = reinterpret_cast<int*>(base + l.status);
+  p.y_obs = nullptr;
+  p.t_noise = static_cast<uint32_t>(s->t + 1);
+  p.ld = chunk;
+  float* slots = reinterpret_cast<float*>(base + l.total);
+  const size_t arr = static_cast<size_t>(s->n) * chunk;  // elements of one staged array
+  const size_t hp = static_cast<size_t>(ld_host) * sizeof(float), dp = static_cast<size_t>(chunk) * sizeof(float);
+
+  long long k = 0;
+  for (long long j0 = 0; j0 < s->d; j0 += chunk, ++k) {
+    const long long w = (s->d - j0 < chunk) ? s->d - j0 : chunk;
+    cudaStream_t st = s->host_stream[k & 1];
+    float* sx = slots + (k & 1) * 5 * arr;
+    float *sy = sx + arr, *sg = sy + arr, *sa = sg + arr, *sc = sa + arr;
+    const size_t wb = static_cast<size_t>(w) * sizeof(float);
+    e = cudaMemcpy2DAsync(sx, dp, x + j0, hp, wb, s->n, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpy2DAsync(sy, dp, y + j0, hp, wb, s->n, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpy2DAsync(sg, dp, g + j0, hp, wb, s->n, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpy2DAsync(sa, dp, a + j0, hp, wb, s->n, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpy2DAsync(sc, dp, c + j0, hp, wb, s->n, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return fail_cuda(s, e, "detag_step_host: host-to-device copy");
+    p.x = sx; p.y = sy; p.g = sg; p.a = sa; p.c = sc;
+    p.d = w;
+    p.coord_offset = s->coord_offset + j0;
+    rc = launch_step(s, p, st);
+    if (rc != DETAG_OK) return rc;
+    e = cudaMemcpy2DAsync(x + j0, hp, sx, dp, wb, s->n, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpy2DAsync(y + j0, hp, sy, dp, wb, s->n, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpy2DAsync(g + j0, hp, sg, dp, wb, s->n, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return fail_cuda(s, e, "detag_step_host: device-to-host copy");
   }
-  if (e != 0) return fail_cuda(s, e, "detag_step launch");
+  for (int q = 0; q < 2 && e == cudaSuccess; ++q) {
+    e = cudaEventRecord(s->host_event[q], s->host_stream[q]);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(user, s->host_event[q], 0);
+  }
+  if (e != cudaSuccess) return fail_cuda(s, e, "detag_step_host: join");
   s->t += 1;
   return DETAG_OK;
 }
@@ -324,6 +431,13 @@ const char* detag_last_error(const detag_state* s) { return s ? s->err.c_str() :
 
 int detag_destroy(detag_state* s) {
   if (!s) return DETAG_ERR_ARG;
+  for (int k = 0; k < 2; ++k)
+    if (s->host_stream[k]) {
+      cudaStreamSynchronize(s->host_stream[k]);
+      cudaStreamDestroy(s->host_stream[k]);
+    }
+  for (int k = 0; k < 3; ++k)
+    if (s->host_event[k]) cudaEventDestroy(s->host_event[k]);
   delete s;
   return DETAG_OK;
 }

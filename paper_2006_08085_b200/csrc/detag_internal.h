@@ -92,6 +92,10 @@ struct detag_state {
   long long coord_offset = 0;
   long long t = 0;
 
+  // host-resident stepping: two internal streams and their events, created on first use
+  cudaStream_t host_stream[2] = {nullptr, nullptr};
+  struct CUevent_st* host_event[3] = {nullptr, nullptr, nullptr};
+
   int device = -1;
   int sm_count = 0;
   int smem_optin = 0;
