@@ -158,6 +158,33 @@ int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* 
 /* Device bytes detag_step_host needs to run with chunks of `chunk_coords` coordinates (a multiple of 128). */
 int detag_host_staging_bytes(const detag_state* s, int64_t chunk_coords, size_t* bytes);
 
+/*
+ * Consensus error (same definition and kernels as detag_consensus_error) for callers that cannot
+ * give the library any scratch memory.  The paper has no counterpart: this entry point exists for
+ * the sake of its callers only.
+ *
+ * Who needs it: code that must not allocate device memory at the point where it wants the number,
+ * and has no workspace at hand either - for example a monitoring hook that runs while a CUDA graph
+ * is being replayed or inside a memory-pool region where cudaMalloc would synchronise the device,
+ * a plug-in that is handed only the model buffer, or a process whose allocator has already given all
+ * device memory to the training job.  It takes no detag_state and no workspace: only the input
+ * x (device, [n][ld] float32, ld >= d) and the output *host_out (host).
+ *
+ * The partial sums go to an array that is compiled into the library (1 MiB + one result slot per
+ * GPU that loads it, held until the process exits), one float64 partial per 256 coordinates.  That
+ * fixes the limit: d <= 33,554,432 (and n <= 1024); larger sizes return DETAG_ERR_UNSUPPORTED and
+ * do nothing.  The call allocates and frees nothing, on the device or through any library.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress) and
+ * caches it; make that first call outside any stream capture.  All calls on a device share the one
+ * array.  Every slot a call reads is written by that call first, so leftovers of earlier calls do
+ * no harm and nothing has to be cleared; but two calls that overlap on the GPU (different streams,
+ * or different host threads) race on it and both results are then garbage: serialise them.
+ * Enqueues on `stream`, waits for it, writes *host_out.
+ * Errors: ARG, UNSUPPORTED (size beyond the built-in array, device ordinal >= 64), CUDA.
+ */
+int detag_consensus_error_static(int n, int64_t d, int64_t ld, const float* x, void* stream, double* host_out);
+
 /* Step counter t (number of completed steps; enters the noise counter).  set_step is for resume. */
 int detag_get_step(const detag_state* s, int64_t* t);
 int detag_set_step(detag_state* s, int64_t t);

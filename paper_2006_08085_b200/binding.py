@@ -57,6 +57,7 @@ SIGNATURES = {
     "detag_step_host": (ctypes.c_int, [_P, ctypes.c_int64, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P]),
     "detag_host_staging_bytes": (ctypes.c_int, [_P, ctypes.c_int64, ctypes.POINTER(ctypes.c_size_t)]),
     "detag_consensus_error": (ctypes.c_int, [_P, _P, _F64P]),
+    "detag_consensus_error_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_int64, ctypes.c_int64, _P, _P, _F64P]),
     "detag_get_step": (ctypes.c_int, [_P, ctypes.POINTER(ctypes.c_int64)]),
     "detag_set_step": (ctypes.c_int, [_P, ctypes.c_int64]),
     "detag_status": (ctypes.c_int, [_P, _P]),
@@ -194,6 +195,15 @@ def detag_consensus_error(state, stream=None) -> float:
     out = ctypes.c_double(float("nan"))
     _check(lib().detag_consensus_error(state, _stream_handle(stream), ctypes.byref(out)), "detag_consensus_error",
            state)
+    return float(out.value)
+
+
+def detag_consensus_error_static(n: int, d: int, ld: int, x, stream=None) -> float:
+    """Consensus error of the device array x ([n][ld] float32) using only the library's built-in scratch
+    array: for callers that cannot allocate device memory or pass a workspace.  d <= 33,554,432."""
+    out = ctypes.c_double(float("nan"))
+    _check(lib().detag_consensus_error_static(int(n), int(d), int(ld), _dev_ptr(x), _stream_handle(stream),
+                                              ctypes.byref(out)), "detag_consensus_error_static")
     return float(out.value)
 
 

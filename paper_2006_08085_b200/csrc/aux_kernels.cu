@@ -117,3 +117,57 @@ int launch_consensus_error(const StepParams& p, double* partials, double* result
 }
 
 }  // namespace detag
+
+// ---------------------------------------------------------------------------------------------------
+// Consensus error without any caller-provided or allocated scratch.
+//
+// The partial sums live in this file-scope device array, which every GPU that loads the library keeps
+// until the process exits (1 MiB + one result slot).  One partial per block of 256 coordinates, so the
+// array bounds the problem size: d <= kStaticMaxCoords.  Host code may not hand the array's NAME to a
+// kernel (on the host it is only a stand-in symbol); the device address is looked up once per device
+// with cudaGetSymbolAddress and cached.
+namespace {
+
+constexpr int kStaticPartials = 131072;                                   // 1 MiB of float64 partial sums
+constexpr long long kStaticMaxCoords = static_cast<long long>(kStaticPartials) * 256;  // 33,554,432
+constexpr int kStaticMaxDevices = 64;
+
+static __device__ __align__(256) double g_static_consensus_scratch[kStaticPartials + 32];
+
+double* g_static_scratch_addr[kStaticMaxDevices] = {nullptr};
+
+}  // namespace
+
+extern "C" int detag_consensus_error_static(int n, int64_t d, int64_t ld, const float* x, void* stream,
+                                            double* host_out) {
+  if (n <= 0 || d <= 0 || ld < d || !x || !host_out) return DETAG_ERR_ARG;
+  if (n > detag::kMaxWorkers || d > kStaticMaxCoords) return DETAG_ERR_UNSUPPORTED;  // beyond the static scratch
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess) return DETAG_ERR_CUDA;
+  if (device < 0 || device >= kStaticMaxDevices) return DETAG_ERR_UNSUPPORTED;
+  if (g_static_scratch_addr[device] == nullptr) {  // first call on this device: resolve the array's device address
+    double* addr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&addr), g_static_consensus_scratch) != cudaSuccess || !addr)
+      return DETAG_ERR_CUDA;
+    g_static_scratch_addr[device] = addr;
+  }
+  double* partials = g_static_scratch_addr[device];
+  double* result = partials + kStaticPartials;
+  detag::StepParams p{};
+  p.n = n;
+  p.d = d;
+  p.ld = ld;
+  p.x = const_cast<float*>(x);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // One CTA per 256 coordinates: every partial slot in [0, grid) is overwritten, and so is the result
+  // slot, so nothing left over from an earlier call is ever read and nothing needs clearing.
+  const int grid = static_cast<int>((d + detag::kAuxThreads - 1) / detag::kAuxThreads);
+  detag::consensus_partial_kernel<<<static_cast<unsigned>(grid), detag::kAuxThreads, 0, st>>>(p, partials);
+  if (cudaGetLastError() != cudaSuccess) return DETAG_ERR_CUDA;
+  detag::consensus_final_kernel<<<1, detag::kAuxThreads, 0, st>>>(partials, grid, result);
+  if (cudaGetLastError() != cudaSuccess) return DETAG_ERR_CUDA;
+  if (cudaMemcpyAsync(host_out, result, sizeof(double), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return DETAG_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return DETAG_ERR_CUDA;
+  return DETAG_OK;
+}
