@@ -101,8 +101,16 @@ StepParams make_params(const detag_state* s) {
   return p;
 }
 
+bool dense_ok(const detag_state* s) {
+  return !s->poly.empty() && s->d <= 0x7fffffffLL && detag::dense_variant_available(s->n);
+}
+
+// Host cost model.  The dense product needs n multiply-adds per element and array against the sparse
+// rounds' K*(nnz per row), but keeps its outputs in registers and needs no barriers; it wins for every
+// n it supports.
 int resolve_variant(const detag_state* s) {
   if (s->variant_forced != DETAG_VARIANT_AUTO) return s->variant_forced;
+  if (dense_ok(s)) return DETAG_VARIANT_DENSE;
   return DETAG_VARIANT_CSR;
 }
 
@@ -122,6 +130,9 @@ int query_device(detag_state* s) {
 int launch_step(detag_state* s, StepParams& p, cudaStream_t stream) {
   int e = 0;
   switch (resolve_variant(s)) {
+    case DETAG_VARIANT_DENSE:
+      e = detag::launch_step_dense(p, s->sm_count, stream);
+      break;
     case DETAG_VARIANT_CSR:
     default: {
       const int rc = detag::plan_step_csr(p, s->smem_optin);
@@ -260,6 +271,8 @@ int detag_set_variant(detag_state* s, int variant) {
     case DETAG_VARIANT_CSR:
       break;
     case DETAG_VARIANT_DENSE:
+      if (!dense_ok(s)) return fail(s, DETAG_ERR_UNSUPPORTED, "detag_set_variant: dense variant needs n <= 64");
+      break;
     case DETAG_VARIANT_RING:
       return fail(s, DETAG_ERR_UNSUPPORTED, "detag_set_variant: variant not available for this matrix");
     default:

@@ -86,8 +86,11 @@ def _check_trajectory(m, K, eta, alpha, a, c, x0, sigma, seed, steps, j0=0, vari
                     errs.pop("x")  # x0 is an input (and may be all zero)
                 assert max(errs.values()) <= bound, (v, t, errs)
             s.status()
-            ce = s.consensus_error()
-            assert ce == pytest.approx(orc.consensus_error(ref[-1][0]), rel=1e-4, abs=1e-12)
+            # consensus error = squared norm of the projection of x off the consensus space, so by the
+            # triangle inequality its root moves by at most ||x_gpu - x_ref||_F
+            ce, ce_ref = s.consensus_error(), orc.consensus_error(ref[-1][0])
+            dist = float(np.sqrt(((s.download("x").astype(np.float64) - ref[-1][0]) ** 2).sum()))
+            assert abs(np.sqrt(ce) - np.sqrt(ce_ref)) <= dist * (1 + 1e-9) + 1e-12 * np.sqrt(ce_ref)
 
 
 # ----------------------------------------------------------------------------- small and edge cases
