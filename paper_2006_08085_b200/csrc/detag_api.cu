@@ -131,7 +131,8 @@ int launch_step(detag_state* s, StepParams& p, cudaStream_t stream) {
   int e = 0;
   switch (resolve_variant(s)) {
     case DETAG_VARIANT_DENSE:
-      e = detag::launch_step_dense(p, s->sm_count, stream);
+      e = p.n <= 32 ? detag::launch_step_mma(p, s->sm_count, stream)
+                    : detag::launch_step_dense(p, s->sm_count, stream);
       break;
     case DETAG_VARIANT_CSR:
     default: {

@@ -333,9 +333,6 @@ int launch_dense(StepParams p, int sm_count, cudaStream_t stream) {
 bool dense_variant_available(int n) { return n >= 1 && n <= kMaxDenseWorkers && encode_tiled_fn() != nullptr; }
 
 int launch_step_dense(const StepParams& p, int sm_count, cudaStream_t stream) {
-  if (p.n <= 8) return launch_dense<8>(p, sm_count, stream);
-  if (p.n <= 16) return launch_dense<16>(p, sm_count, stream);
-  if (p.n <= 32) return launch_dense<32>(p, sm_count, stream);
   return launch_dense<64>(p, sm_count, stream);
 }
 
