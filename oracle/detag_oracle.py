@@ -26,7 +26,7 @@ and counter (j low word, j high word, i // 4, t) yields four words r0..r3; the p
 4q+3 (q = i // 4) by the Box-Muller transform with
 
     u_rad = ((r_even >> 9) + 0.5) * 2^-23   in (0, 1)
-    u_ang = (r_odd >> 8) * 2^-24            in [0, 1)
+    u_ang = (r_odd >> 9) * 2^-23            in [0, 1)
     rad = sqrt(-2 ln u_rad) ;  first = rad*cos(2 pi u_ang) ;  second = rad*sin(2 pi u_ang).
 """
 from __future__ import annotations
@@ -105,7 +105,7 @@ def standard_normal_noise(seed: int, t: int, n: int, j0: int, j1: int) -> np.nda
     out = np.empty((nq * 4, m), dtype=np.float64)
     for p in range(2):
         u_rad = ((r[2 * p] >> np.uint32(9)).astype(np.float64) + 0.5) * 2.0 ** -23
-        u_ang = (r[2 * p + 1] >> np.uint32(8)).astype(np.float64) * 2.0 ** -24
+        u_ang = (r[2 * p + 1] >> np.uint32(9)).astype(np.float64) * 2.0 ** -23
         rad = np.sqrt(-2.0 * np.log(u_rad))
         out[2 * p::4] = rad * np.cos(2.0 * math.pi * u_ang)
         out[2 * p + 1::4] = rad * np.sin(2.0 * math.pi * u_ang)

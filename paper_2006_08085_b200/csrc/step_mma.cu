@@ -12,7 +12,7 @@
 // Row permutation: block t of P holds workers {4r + t : r = 0..7}, so lane (r = lane/4) ends up with
 // workers 4r..4r+3 - exactly the four workers one Philox call serves - for its two coordinates.
 //
-// Data movement: a producer warp fills two stages with bulk asynchronous copies, one 512-byte row per
+// Data movement: a producer warp fills three stages with bulk asynchronous copies, one 384-byte row per
 // (array, worker) and lane, completion counted on the stage's "full" mbarrier.  Rows are laid out with
 // a padded pitch (S+8 floats for x, y; S+4 for g, a, c) so the B-fragment loads are bank-conflict free.
 // Consumer warps hand a stage back with one arrive per warp on its "empty" mbarrier.  Results go to
@@ -28,13 +28,13 @@ namespace detag {
 namespace {
 
 constexpr int kN = 32;           // padded worker count
-constexpr int kS = 128;          // coordinates per stage
+constexpr int kS = 96;           // coordinates per stage: 12 tiles of 8, one per consumer warp
 constexpr int kPitchXY = kS + 8; // floats; 8 mod 32 -> the four workers of a B fragment hit disjoint banks
 constexpr int kPitchE = kS + 4;  // floats; rows of g, a, c (read in the accumulator layout)
 constexpr int kStageFloats = 2 * kN * kPitchXY + 3 * kN * kPitchE;
 constexpr int kStageBytes = kStageFloats * 4;
-constexpr int kMmaStages = 2;
-constexpr int kConsumerWarps = 8;
+constexpr int kMmaStages = 3;
+constexpr int kConsumerWarps = 12;
 constexpr int kMmaThreads = (kConsumerWarps + 1) * 32;
 constexpr int kTilesPerStage = kS / 8;
 constexpr unsigned kMmaSpinLimit = 1u << 22;
