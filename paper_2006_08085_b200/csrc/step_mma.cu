@@ -4,41 +4,63 @@
 // Algorithm 3.  For a slab of coordinates the step is therefore two small dense contractions
 // (P times the tracker rows, P times the model rows) followed by Algorithm 2's element-wise updates.
 // Here the contractions run as warp-level float64 matrix multiply-accumulates (mma m8n8k4, f64):
-//   A (8 x 4) : a block of P.  All 4 x 8 blocks of the 32 x 32 matrix stay in registers for the
-//               whole kernel (32 doubles per lane).
+//   A (8 x 4) : a block of P.  The 4 x 8 blocks of the 32 x 32 matrix sit in shared memory in
+//               fragment order (one conflict-free 8-byte load per lane and block).
 //   B (4 x 8) : four workers x eight coordinates of the staged tracker / model slab, read from shared
 //               memory once per warp (one 4-byte load + one widening per lane and block).
 //   C (8 x 8) : float64 accumulators, 2 per lane and block.
 // Row permutation: block t of P holds workers {4r + t : r = 0..7}, so lane (r = lane/4) ends up with
 // workers 4r..4r+3 - exactly the four workers one Philox call serves - for its two coordinates.
 //
-// Data movement: a producer warp fills three stages with bulk asynchronous copies, one 384-byte row per
-// (array, worker) and lane, completion counted on the stage's "full" mbarrier.  Rows are laid out with
-// a padded pitch (S+8 floats for x, y; S+4 for g, a, c) so the B-fragment loads are bank-conflict free.
-// Consumer warps hand a stage back with one arrive per warp on its "empty" mbarrier.  Results go to
-// global memory straight from the accumulator layout (32-byte row segments, whole sectors).
+// Warp roles of the persistent CTA (one per SM):
+//   producer  one thread keeps three input stages in flight with five 2-D TMA tile loads each (all 32
+//             worker rows x one slab of 64 coordinates of x, y, g, a, c), completion counted on the
+//             stage's "full" mbarrier.  The tiles are loaded a few columns wider than the slab (72 for
+//             x, y; 68 for g, a, c): TMA writes a tile densely, so the box width IS the row pitch in
+//             shared memory, and 8 (mod 32) floats makes the B-fragment loads bank-conflict free.  The
+//             extra columns belong to the next slab (read by its CTA at about the same time, so they
+//             come from L2) and are not used.
+//   consumers 16 warps in two groups that take alternate slabs; a warp owns 8 coordinates of the slab:
+//             64 MMAs, then the element-wise tail (model update, Philox/Box-Muller noise, gradient,
+//             tracker fold), results written to the group's dense output tile in shared memory.
+//   storer    one thread writes each finished output tile (x', y', g': 32 rows x 256 bytes) with three
+//             TMA tile stores.  Row-contiguous 256-byte writes matter: storing straight from the
+//             accumulator layout (32-byte pieces of 8 rows per instruction) halves the HBM throughput.
 // Every mbarrier wait is bounded; a wait that gives up sets the status word and the CTA winds down.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "detag_internal.h"
 #include "noise.cuh"
+#include "tma.cuh"
 
 namespace detag {
 
 namespace {
 
-constexpr int kN = 32;           // padded worker count
-constexpr int kS = 96;           // coordinates per stage: 12 tiles of 8, one per consumer warp
-constexpr int kPitchXY = kS + 8; // floats; 8 mod 32 -> the four workers of a B fragment hit disjoint banks
-constexpr int kPitchE = kS + 4;  // floats; rows of g, a, c (read in the accumulator layout)
+constexpr int kN = 32;            // padded worker count
+constexpr int kS = 64;            // coordinates per slab: 8 tiles of 8, one per consumer warp of a group
+constexpr int kPitchXY = kS + 8;  // floats; 8 mod 32 -> the four workers of a B fragment hit disjoint banks
+constexpr int kPitchE = kS + 4;   // floats; rows of g, a, c (read in the accumulator layout)
 constexpr int kStageFloats = 2 * kN * kPitchXY + 3 * kN * kPitchE;
 constexpr int kStageBytes = kStageFloats * 4;
 constexpr int kMmaStages = 3;
-constexpr int kConsumerWarps = 12;
-constexpr int kMmaThreads = (kConsumerWarps + 1) * 32;
-constexpr int kTilesPerStage = kS / 8;
-constexpr unsigned kMmaSpinLimit = 1u << 22;
-constexpr size_t kMmaSmemBytes = 128 + static_cast<size_t>(kMmaStages) * kStageBytes + 64;
+constexpr int kWarpGroups = 2;    // consumer groups take alternate slabs, so their phases interleave
+constexpr int kGroupWarps = kS / 8;
+constexpr int kConsumerWarps = kGroupWarps * kWarpGroups;
+constexpr int kProducerWarp = kConsumerWarps, kStoreWarp = kConsumerWarps + 1;
+constexpr int kMmaThreads = (kConsumerWarps + 2) * 32;
+constexpr int kOutFloats = 3 * kN * kS;       // x', y', g' tiles of one slab, dense rows
+constexpr int kFragBytes = 32 * 32 * 8;       // P in fragment order
+constexpr unsigned kMmaSpinLimit = 1u << 20;  // polls before a wait gives up (each may suspend ~kSuspendHintNs)
+constexpr unsigned kSuspendHintNs = 2000;
+constexpr size_t kMmaSmemBytes =
+    static_cast<size_t>(kMmaStages) * kStageBytes + kWarpGroups * kOutFloats * 4 + kFragBytes + 128;
+
+struct MmaMaps {
+  CUtensorMap x, y, g, a, c;  // loads (padded boxes)
+  CUtensorMap xs, ys, gs;     // stores (exact slab width)
+};
 
 __device__ __forceinline__ uint32_t s_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
@@ -48,20 +70,36 @@ __device__ __forceinline__ bool bar_wait(uint64_t* bar, unsigned parity) {
     unsigned done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done)
-        : "r"(addr), "r"(parity)
+        : "r"(addr), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     if (done) return true;
   }
   return false;
 }
 
-__device__ __forceinline__ void bulk_row(float* dst, const float* src, unsigned bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   s_addr(dst)),
-               "l"(src), "r"(bytes), "r"(s_addr(bar))
+__device__ __forceinline__ void bar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_addr(bar)) : "memory");
+}
+
+__device__ __forceinline__ void bar_init(uint64_t* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_addr(bar)), "r"(count));
+}
+
+__device__ __forceinline__ void tile_load(float* dst, const CUtensorMap* map, int col, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          s_addr(dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(col), "r"(0), "r"(s_addr(bar))
+      : "memory");
+}
+
+__device__ __forceinline__ void tile_store(const CUtensorMap* map, int col, const float* src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+                   reinterpret_cast<uint64_t>(map)),
+               "r"(col), "r"(0), "r"(s_addr(src))
                : "memory");
 }
 
@@ -71,91 +109,124 @@ __device__ __forceinline__ void dmma(double (&c)[2], double a, double b) {
                : "d"(a), "d"(b));
 }
 
-__global__ void __launch_bounds__(kMmaThreads, 1) step_mma_kernel(const StepParams p) {
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
-  float* stage_mem = reinterpret_cast<float*>(base);
-  uint64_t* full = reinterpret_cast<uint64_t*>(base + static_cast<size_t>(kMmaStages) * kStageBytes);
+__global__ void __launch_bounds__(kMmaThreads, 1)
+step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
+  // No static shared memory in this kernel: the dynamic array starts at the CTA's shared window, whose
+  // 128-byte alignment (needed by the TMA tiles) is checked below rather than assumed.
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  float* stage_mem = reinterpret_cast<float*>(smem_raw);
+  float* out_mem = stage_mem + kMmaStages * kStageFloats;                             // [group][x', y', g'][32][kS]
+  double* frag = reinterpret_cast<double*>(out_mem + kWarpGroups * kOutFloats);       // [t][ks][lane]
+  uint64_t* full = reinterpret_cast<uint64_t*>(frag + 32 * 32);
   uint64_t* empty = full + kMmaStages;
+  uint64_t* out_ready = empty + kMmaStages;      // [group]: the group's 8 warps have written their outputs
+  uint64_t* out_free = out_ready + kWarpGroups;  // [group]: the stores have finished reading the tile
+  if ((s_addr(smem_raw) & 127u) != 0) {
+    if (threadIdx.x == 0) atomicExch(p.status, 2);
+    return;
+  }
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = p.n;
-  // rows >= n and slab tails are never written by the copies: give them a finite value once
-  for (int e = tid; e < kMmaStages * kStageFloats; e += kMmaThreads) stage_mem[e] = 0.f;
+  // P in fragment order: block (t, ks), lane (r, kq) holds P[4r + t][4ks + kq]
+  for (int e = tid; e < 32 * 32; e += kMmaThreads) {
+    const int l = e & 31, ks = (e >> 5) & 7, t = e >> 8;
+    const int i = 4 * (l >> 2) + t, j = 4 * ks + (l & 3);
+    frag[e] = (i < n && j < n) ? p.poly[static_cast<size_t>(i) * n + j] : 0.0;
+  }
   if (tid == 0) {
     for (int s = 0; s < kMmaStages; ++s) {
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_addr(&full[s])), "r"(1));
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_addr(&empty[s])), "r"(kConsumerWarps));
+      bar_init(&full[s], 1);
+      bar_init(&empty[s], kGroupWarps);
+    }
+    for (int g = 0; g < kWarpGroups; ++g) {
+      bar_init(&out_ready[g], kGroupWarps);
+      bar_init(&out_free[g], 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // the zero fill above went through the generic proxy; order it before the async-proxy copies
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
 
   const long long first = blockIdx.x, stride = gridDim.x;
 
-  if (warp == kConsumerWarps) {
-    // ---------------------------------------------------------------- producer warp: lane = worker row
-    int issued = 0;
-    bool ok = true;
-    for (long long slab = first; slab < p.num_slabs; slab += stride, ++issued) {
-      const int s = issued % kMmaStages;
-      if (issued >= kMmaStages) {
-        if (lane == 0) ok = bar_wait(&empty[s], ((issued / kMmaStages) - 1) & 1);
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      }
-      if (!ok) break;
-      const long long j0 = slab * kS;
-      const long long width = (p.d - j0 < kS) ? p.d - j0 : kS;
-      const unsigned row_bytes = static_cast<unsigned>((width + 3) / 4 * 16);  // ld >= d rounded up to 4: in bounds
-      if (lane == 0) {
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_addr(&full[s])),
-                     "r"(row_bytes * 5u * static_cast<unsigned>(n))
-                     : "memory");
-      }
-      __syncwarp();
-      if (lane < n) {
+  if (warp == kProducerWarp) {
+    // ---------------------------------------------------------------- producer: one elected thread
+    if (lane == 0) {
+      int issued = 0;
+      bool ok = true;
+      for (long long slab = first; slab < p.num_slabs; slab += stride, ++issued) {
+        const int s = issued % kMmaStages;
+        if (issued >= kMmaStages) ok = bar_wait(&empty[s], ((issued / kMmaStages) - 1) & 1);
+        if (!ok) break;
         float* st = stage_mem + static_cast<size_t>(s) * kStageFloats;
-        const long long off = static_cast<long long>(lane) * p.ld + j0;
-        bulk_row(st + lane * kPitchXY, p.x + off, row_bytes, &full[s]);
-        bulk_row(st + kN * kPitchXY + lane * kPitchXY, p.y + off, row_bytes, &full[s]);
+        const int col = static_cast<int>(slab * kS);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_addr(&full[s])),
+                     "r"(static_cast<unsigned>(kStageBytes))
+                     : "memory");
+        tile_load(st, &maps.x, col, &full[s]);
+        tile_load(st + kN * kPitchXY, &maps.y, col, &full[s]);
         float* se = st + 2 * kN * kPitchXY;
-        bulk_row(se + lane * kPitchE, p.g + off, row_bytes, &full[s]);
-        bulk_row(se + kN * kPitchE + lane * kPitchE, p.a + off, row_bytes, &full[s]);
-        bulk_row(se + 2 * kN * kPitchE + lane * kPitchE, p.c + off, row_bytes, &full[s]);
+        tile_load(se, &maps.g, col, &full[s]);
+        tile_load(se + kN * kPitchE, &maps.a, col, &full[s]);
+        tile_load(se + 2 * kN * kPitchE, &maps.c, col, &full[s]);
+      }
+      if (!ok) {
+        atomicExch(p.status, 1);
+        for (int back = 1; back <= kMmaStages && back <= issued; ++back) {  // drain copies still in flight (bounded)
+          const int k = issued - back;
+          bar_wait(&full[k % kMmaStages], (k / kMmaStages) & 1);
+        }
       }
     }
-    if (!ok && lane == 0) {
-      atomicExch(p.status, 1);
-      for (int back = 1; back <= kMmaStages && back <= issued; ++back) {  // drain copies still in flight (bounded)
-        const int k = issued - back;
-        bar_wait(&full[k % kMmaStages], (k / kMmaStages) & 1);
+    return;
+  }
+
+  if (warp == kStoreWarp) {
+    // ---------------------------------------------------------------- storer: one elected thread
+    if (lane == 0) {
+      long long k = 0;
+      for (long long slab = first; slab < p.num_slabs; slab += stride, ++k) {
+        const int g = static_cast<int>(k % kWarpGroups);
+        if (!bar_wait(&out_ready[g], (k / kWarpGroups) & 1)) {
+          atomicExch(p.status, 1);
+          break;
+        }
+        const float* ob = out_mem + g * kOutFloats;
+        const int col = static_cast<int>(slab * kS);
+        if (col < (p.d & ~3LL)) {
+          tile_store(&maps.xs, col, ob);
+          tile_store(&maps.ys, col, ob + kN * kS);
+          tile_store(&maps.gs, col, ob + 2 * kN * kS);
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // the tile may be overwritten now
+        bar_arrive(&out_free[g]);
       }
+      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // all global writes done before the CTA leaves
     }
     return;
   }
 
   // ------------------------------------------------------------------ consumer warps
   const int r = lane >> 2, kq = lane & 3;
-  // A fragments: block (t, s) element [r][kq] = P[4r + t][4s + kq]
-  double afrag[4][8];
-#pragma unroll
-  for (int t = 0; t < 4; ++t)
-#pragma unroll
-    for (int s = 0; s < 8; ++s) {
-      const int i = 4 * r + t, j = 4 * s + kq;
-      afrag[t][s] = (i < n && j < n) ? p.poly[static_cast<size_t>(i) * n + j] : 0.0;
-    }
+  const int group = warp / kGroupWarps, tile = warp % kGroupWarps;
   const double alpha = p.alpha;
   const float sigma = static_cast<float>(p.sigma);
   const bool noisy = p.sigma != 0.0;
+  float* ob = out_mem + group * kOutFloats;
+  const int cl = tile * 8;
+  const long long d_tma = p.d & ~3LL;  // columns below this are written by the TMA stores
 
-  int k = 0;
-  for (long long slab = first; slab < p.num_slabs; slab += stride, ++k) {
-    const int s = k % kMmaStages;
+  long long use = 0;  // how many slabs this group has taken so far
+  for (long long k = group, slab = first + group * stride; slab < p.num_slabs;
+       slab += kWarpGroups * stride, k += kWarpGroups, ++use) {
+    const int s = static_cast<int>(k % kMmaStages);
     bool ok = true;
-    if (lane == 0) ok = bar_wait(&full[s], (k / kMmaStages) & 1);
+    if (lane == 0) {
+      ok = bar_wait(&full[s], (k / kMmaStages) & 1);
+      if (ok && use > 0) ok = bar_wait(&out_free[group], (use - 1) & 1);  // previous tile of this group stored
+    }
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     if (!ok) {
       if (lane == 0) atomicExch(p.status, 1);
@@ -168,9 +239,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) step_mma_kernel(const StepPara
     const float* sc = sa + kN * kPitchE;
     const long long j0 = slab * kS;
 
-    for (int tile = warp; tile < kTilesPerStage; tile += kConsumerWarps) {
-      const int cl = tile * 8;
-      if (j0 + cl >= p.d) break;
+    if (j0 + cl < p.d) {
       double cy[4][2], cx[4][2];
 #pragma unroll
       for (int t = 0; t < 4; ++t) cy[t][0] = cy[t][1] = cx[t][0] = cx[t][1] = 0.0;
@@ -181,8 +250,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) step_mma_kernel(const StepPara
         const double bx = static_cast<double>(sx[src]);
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-          dmma(cy[t], afrag[t][ks], by);
-          dmma(cx[t], afrag[t][ks], bx);
+          const double a = frag[(t * 8 + ks) * 32 + lane];
+          dmma(cy[t], a, by);
+          dmma(cx[t], a, bx);
         }
       }
       // element-wise tail: workers 4r..4r+3 (index t), coordinates j, j+1
@@ -197,7 +267,6 @@ __global__ void __launch_bounds__(kMmaThreads, 1) step_mma_kernel(const StepPara
           xi[e][0] = xi[e][1] = xi[e][2] = xi[e][3] = 0.f;
         }
       }
-      const bool in0 = j < p.d, in1 = j + 1 < p.d;
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const int row = 4 * r + t;
@@ -205,14 +274,13 @@ __global__ void __launch_bounds__(kMmaThreads, 1) step_mma_kernel(const StepPara
         const float2 gv = *reinterpret_cast<const float2*>(sg + eoff);
         const float2 av = *reinterpret_cast<const float2*>(sa + eoff);
         const float2 cv = *reinterpret_cast<const float2*>(sc + eoff);
-        float2 xo, yo, go, yg;
+        float2 xo, yo, go;
         {
           const float x_new = static_cast<float>(fma(-alpha, cy[t][0], cx[t][0]));
           const float g_new = fmaf(av.x, x_new - cv.x, sigma * xi[0][t]);
           xo.x = x_new;
           go.x = g_new;
           yo.x = static_cast<float>(cy[t][0] + (static_cast<double>(g_new) - static_cast<double>(gv.x)));
-          yg.x = static_cast<float>(cy[t][0]);
         }
         {
           const float x_new = static_cast<float>(fma(-alpha, cy[t][1], cx[t][1]));
@@ -220,33 +288,60 @@ __global__ void __launch_bounds__(kMmaThreads, 1) step_mma_kernel(const StepPara
           xo.y = x_new;
           go.y = g_new;
           yo.y = static_cast<float>(cy[t][1] + (static_cast<double>(g_new) - static_cast<double>(gv.y)));
-          yg.y = static_cast<float>(cy[t][1]);
         }
-        if (row < n) {
+        const int ooff = row * kS + cl + 2 * kq;
+        *reinterpret_cast<float2*>(ob + ooff) = xo;
+        *reinterpret_cast<float2*>(ob + kN * kS + ooff) = yo;
+        *reinterpret_cast<float2*>(ob + 2 * kN * kS + ooff) = go;
+        if (j >= d_tma && row < n) {
+          // TMA clips a store at 16-byte granularity; the last d % 4 coordinates are written here so that
+          // nothing beyond column d is touched
           const long long off = static_cast<long long>(row) * p.ld + j;
-          if (in1) {
-            *reinterpret_cast<float2*>(p.x + off) = xo;
-            *reinterpret_cast<float2*>(p.y + off) = yo;
-            *reinterpret_cast<float2*>(p.g + off) = go;
-            if (p.y_obs != nullptr) *reinterpret_cast<float2*>(p.y_obs + off) = yg;
-          } else if (in0) {
+          if (j < p.d) {
             p.x[off] = xo.x;
             p.y[off] = yo.x;
             p.g[off] = go.x;
-            if (p.y_obs != nullptr) p.y_obs[off] = yg.x;
+          }
+          if (j + 1 < p.d) {
+            p.x[off + 1] = xo.y;
+            p.y[off + 1] = yo.y;
+            p.g[off + 1] = go.y;
+          }
+        }
+        if (p.y_obs != nullptr && row < n) {  // optional observer: the gossiped tracker, stored directly
+          const long long off = static_cast<long long>(row) * p.ld + j;
+          if (j + 1 < p.d) {
+            *reinterpret_cast<float2*>(p.y_obs + off) =
+                make_float2(static_cast<float>(cy[t][0]), static_cast<float>(cy[t][1]));
+          } else if (j < p.d) {
+            p.y_obs[off] = static_cast<float>(cy[t][0]);
           }
         }
       }
     }
+    // outputs visible to the TMA store, input stage no longer read by this warp
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
-    if (lane == 0)
-      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_addr(&empty[s])) : "memory");
+    if (lane == 0) {
+      bar_arrive(&out_ready[group]);
+      bar_arrive(&empty[s]);
+    }
   }
 }
 
 }  // namespace
 
 int launch_step_mma(StepParams p, int sm_count, cudaStream_t stream) {
+  MmaMaps maps;
+  if (!make_map(&maps.x, p.x, p.n, p.d, p.ld, kN, kPitchXY) || !make_map(&maps.y, p.y, p.n, p.d, p.ld, kN, kPitchXY) ||
+      !make_map(&maps.g, p.g, p.n, p.d, p.ld, kN, kPitchE) || !make_map(&maps.a, p.a, p.n, p.d, p.ld, kN, kPitchE) ||
+      !make_map(&maps.c, p.c, p.n, p.d, p.ld, kN, kPitchE) || false)
+    return static_cast<int>(cudaErrorInvalidValue);
+  const long long d_tma = p.d & ~3LL;  // the stores' tensor ends on a 16-byte boundary (see the kernel's tail)
+  if (d_tma > 0 && (!make_map(&maps.xs, p.x, p.n, d_tma, p.ld, kN, kS) || !make_map(&maps.ys, p.y, p.n, d_tma, p.ld, kN, kS) ||
+                    !make_map(&maps.gs, p.g, p.n, d_tma, p.ld, kN, kS)))
+    return static_cast<int>(cudaErrorInvalidValue);
+  if (d_tma == 0) maps.xs = maps.ys = maps.gs = maps.x;  // never used: every slab lies beyond column 0
   p.S = kS;
   p.num_slabs = (p.d + kS - 1) / kS;
   cudaError_t e = cudaFuncSetAttribute(step_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -254,7 +349,7 @@ int launch_step_mma(StepParams p, int sm_count, cudaStream_t stream) {
   if (e != cudaSuccess) return static_cast<int>(e);
   const long long grid = p.num_slabs < sm_count ? p.num_slabs : sm_count;
   if (grid <= 0) return 0;
-  step_mma_kernel<<<static_cast<unsigned>(grid), kMmaThreads, kMmaSmemBytes, stream>>>(p);
+  step_mma_kernel<<<static_cast<unsigned>(grid), kMmaThreads, kMmaSmemBytes, stream>>>(p, maps);
   return static_cast<int>(cudaGetLastError());
 }
 
