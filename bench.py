@@ -158,7 +158,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     import torch
     import torch.distributed as dist
 
-    from paper_2006_08085_b200 import binding as B, build
+    from paper_2006_08085_b200 import binding as B, build, sharding
     from paper_2006_08085_b200.session import Session
 
     build.build()
@@ -180,7 +180,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     inputs.objective_data(cfg, threads=threads,
                           out=tuple(host[k].numpy()[:, : cfg.d] for k in ("a", "c", "x")))
     s = Session(m, cfg.d, cfg.K, float("nan"), cfg.alpha, None, None, None, cfg.sigma, cfg.seed,
-                coord_offset=rank * cfg.d, ld=ld, device=str(dev))
+                coord_offset=sharding.weak_scaling_offset(cfg.d, rank), ld=ld, device=str(dev))
     for k in ("a", "c", "x"):
         getattr(s, k).copy_(host[k], non_blocking=True)
     torch.cuda.synchronize(dev)
@@ -214,11 +214,8 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     s.status()
     total_ms = events[0].elapsed_time(events[-1])
     per_step = np.array([events[k].elapsed_time(events[k + 1]) for k in range(args.steps)])
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms_max = float(t.item())
-    consensus = s.consensus_error()
+    total_ms_max = sharding.reduce_max(total_ms, dist if world > 1 else None, dev)
+    consensus = sharding.reduce_sum(s.consensus_error(), dist if world > 1 else None, dev)
 
     # ---- end to end through the host-buffer entry point: H2D of x, y, g, a, c and D2H of x, y, g every step
     e2e = None
@@ -250,10 +247,8 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
             host_step()
         e1.record(stream)
         torch.cuda.synchronize(dev)
-        te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * cfg.wc * e_steps / (float(te.item()) * 1e-3), "unit": UNIT,
+        te = sharding.reduce_max(e0.elapsed_time(e1), dist if world > 1 else None, dev)
+        e2e = {"value": world * cfg.wc * e_steps / (te * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": 5 * 4 * cfg.wc, "d2h_bytes_per_step": 3 * 4 * cfg.wc, "steps": e_steps,
                "api": "detag_step_host (page-locked host state; chunked copy/step/copy on two streams)"}
         del staging

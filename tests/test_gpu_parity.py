@@ -240,3 +240,65 @@ def test_consensus_error_matches_definition():
     cons = np.tile(rng.standard_normal((1, 1000)).astype(np.float32), (16, 1))
     with Session(m, 1000, 2, 0.1, 0.1, a[:, :1000], a[:, :1000], cons) as s:
         assert s.consensus_error() == 0.0
+
+
+# ----------------------------------------------------------------------------- full size, bench launch configuration
+def _full_size_sampled(name, blocks, steps):
+    """The config at its full size and in the launch configuration bench.py times (default variant, no observer).
+
+    The oracle cannot run 8e8 elements, but the step never mixes coordinates: sampled coordinate blocks are
+    recomputed by the oracle on their own (global column offset in the noise counter) and compared element by
+    element after one step and in relative L2 over the config's trajectory.
+    """
+    import os
+
+    cfg = inputs.CONFIGS[name]
+    m = inputs.gossip_matrix(cfg)
+    eta = orc.spectrum(m.to_dense()).eta
+    with Session(m, cfg.d, cfg.K, eta, cfg.alpha, None, None, None, cfg.sigma, cfg.seed) as s:
+        chunk = 1 << 21
+        for j0 in range(0, cfg.d, chunk):  # objective data, chunk by chunk (bounded host memory)
+            j1 = min(cfg.d, j0 + chunk)
+            a, c, x0 = inputs.objective_data(cfg, j0, j1, threads=min(16, os.cpu_count() or 1))
+            for nm, host in (("a", a), ("c", c), ("x", x0)):
+                getattr(s, nm)[:, j0:j1].copy_(s.torch.from_numpy(host))
+        s.init()
+        refs = []
+        for (j0, w) in blocks:
+            a, c, x0 = inputs.objective_data(cfg, j0, j0 + w)
+            p = oracle_problem(m, cfg.K, eta, cfg.alpha, a, c, cfg.sigma, cfg.seed, j0)
+            (x32, y32, g32), one = one_step_from_rounded_state(p, x0)
+            # the initial state the GPU computed itself, against the oracle's (relative L2: it is rounded storage)
+            assert rel_l2(s.g[:, j0:j0 + w].cpu().numpy(), g32.astype(np.float64)) < 1e-6
+            for nm, host in (("x", x32), ("y", y32), ("g", g32)):  # same float32 start on both sides
+                getattr(s, nm)[:, j0:j0 + w].copy_(s.torch.from_numpy(host))
+            traj = []
+            orc.run(p, x0, steps, observe=lambda st: traj.append((st.x.copy(), orc.folded_tracker(st), st.g_new.copy())))
+            refs.append((j0, w, one, traj))
+        for t in range(1, steps + 1):
+            s.step()
+            for (j0, w, one, traj) in refs:
+                got = {k: getattr(s, k)[:, j0:j0 + w].cpu().numpy() for k in ("x", "y", "g")}
+                if t == 1:
+                    x_ref, _, g_ref, yf_ref = one
+                    r = {"x": worst_ratio(got["x"], x_ref), "g": worst_ratio(got["g"], g_ref),
+                         "y": worst_ratio(got["y"], yf_ref, extra=HALF_ULP32 * np.abs(g_ref))}
+                    assert max(r.values()) <= 1.0, (name, j0, r)
+                errs = {k: rel_l2(got[k], ref) for k, ref in zip(("x", "y", "g"), traj[t])}
+                assert max(errs.values()) <= 1e-4, (name, j0, t, errs)
+        s.status()
+
+
+def test_cfg5_full_size_sampled_blocks():
+    d = inputs.CONFIGS["cfg5"].d
+    _full_size_sampled("cfg5", [(0, 512), (64 * 12345 + 8, 300), (d // 2 - 100, 333), (d - 640, 640)], steps=20)
+
+
+def test_cfg4_full_size_sampled_blocks():
+    d = inputs.CONFIGS["cfg4"].d
+    _full_size_sampled("cfg4", [(0, 64), (500_001, 50), (d - 40, 40)], steps=50)
+
+
+def test_cfg3_full_size_sampled_blocks():
+    d = inputs.CONFIGS["cfg3"].d
+    _full_size_sampled("cfg3", [(0, 128), (7_000_003, 96), (d - 128, 128)], steps=10)
