@@ -59,7 +59,7 @@ enum {
   DETAG_VARIANT_AUTO = 0,  /* host cost model picks */
   DETAG_VARIANT_CSR = 1,   /* K rounds of neighbour-indexed sums over the CSR rows, slab staged on chip */
   DETAG_VARIANT_DENSE = 2, /* one product with the host-precomputed polynomial P_K(M), n <= 64 */
-  DETAG_VARIANT_RING = 3   /* K rounds with register-blocked halo exchange, circulant ring matrices only */
+  DETAG_VARIANT_RING = 3   /* banded circulant polynomial P_K(M): circulant M (rings), n % 32 == 0, n >= 64, K*bandwidth <= 16 */
 };
 
 /*

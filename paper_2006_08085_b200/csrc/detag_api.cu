@@ -74,6 +74,48 @@ void gossip_polynomial(const detag_state* s, std::vector<double>& out) {
   out = cur;
 }
 
+// Circulant M (row i = row 0 shifted by i): then P_K(M) is circulant too; its row 0 is computed with the
+// recursion of Algorithm 3 on a single row and stored as a band around the diagonal.
+void analyse_circulant(detag_state* s) {
+  const int n = s->n;
+  std::vector<double> row0(n, 0.0);
+  for (int k = s->row_ptr[0]; k < s->row_ptr[1]; ++k) row0[s->col_idx[k]] = s->vals[k];
+  for (int i = 1; i < n; ++i) {
+    if (s->row_ptr[i + 1] - s->row_ptr[i] != s->row_ptr[1] - s->row_ptr[0]) return;
+    for (int k = s->row_ptr[i]; k < s->row_ptr[i + 1]; ++k)
+      if (s->vals[k] != row0[((s->col_idx[k] - i) % n + n) % n]) return;
+  }
+  s->circulant = true;
+  // row 0 of P_r: q_{r+1}[j] = (1+eta) sum_k M[0][k] q_r[(j - k) mod n] - eta q_{r-1}[j]   (circulant product)
+  std::vector<double> prev(n, 0.0), cur, next(n);
+  prev[0] = 1.0;
+  cur = prev;
+  for (int r = 0; r < s->K; ++r) {
+    for (int j = 0; j < n; ++j) {
+      double acc = 0.0;
+      for (int k = s->row_ptr[0]; k < s->row_ptr[1]; ++k)
+        acc += s->vals[k] * cur[((j - s->col_idx[k]) % n + n) % n];
+      next[j] = (1.0 + s->eta) * acc - s->eta * prev[j];
+    }
+    prev.swap(cur);
+    cur.swap(next);
+  }
+  int hb = 0;
+  for (int j = 0; j < n; ++j)
+    if (cur[j] != 0.0) {
+      const int delta = j <= n / 2 ? j : n - j;
+      if (delta > hb) hb = delta;
+    }
+  s->half_band = hb;
+  if (hb <= 16 && n >= 2 * hb + 1)
+    for (int delta = -16; delta <= 16; ++delta)
+      s->band[delta + 16] = (delta >= -hb && delta <= hb) ? cur[((delta % n) + n) % n] : 0.0;
+}
+
+bool band_ok(const detag_state* s) {
+  return s->circulant && s->d <= 0x7fffffffLL && detag::band_variant_available(s->n, s->half_band);
+}
+
 StepParams make_params(const detag_state* s) {
   StepParams p{};
   p.n = s->n;
@@ -111,6 +153,7 @@ bool dense_ok(const detag_state* s) {
 int resolve_variant(const detag_state* s) {
   if (s->variant_forced != DETAG_VARIANT_AUTO) return s->variant_forced;
   if (dense_ok(s)) return DETAG_VARIANT_DENSE;
+  if (band_ok(s)) return DETAG_VARIANT_RING;
   return DETAG_VARIANT_CSR;
 }
 
@@ -133,6 +176,9 @@ int launch_step(detag_state* s, StepParams& p, cudaStream_t stream) {
     case DETAG_VARIANT_DENSE:
       e = p.n <= 32 ? detag::launch_step_mma(p, s->sm_count, stream)
                     : detag::launch_step_dense(p, s->sm_count, stream);
+      break;
+    case DETAG_VARIANT_RING:
+      e = detag::launch_step_band(p, s->band, s->sm_count, stream);
       break;
     case DETAG_VARIANT_CSR:
     default: {
@@ -190,6 +236,7 @@ int detag_create(detag_state** out, int n, int64_t d, const int32_t* row_ptr, co
   s->col_idx.assign(col_idx, col_idx + nnz);
   s->vals.assign(vals, vals + nnz);
   if (n <= detag::kMaxDenseWorkers) gossip_polynomial(s, s->poly);
+  analyse_circulant(s);
   *out = s;
   return DETAG_OK;
 }
@@ -275,7 +322,10 @@ int detag_set_variant(detag_state* s, int variant) {
       if (!dense_ok(s)) return fail(s, DETAG_ERR_UNSUPPORTED, "detag_set_variant: dense variant needs n <= 64");
       break;
     case DETAG_VARIANT_RING:
-      return fail(s, DETAG_ERR_UNSUPPORTED, "detag_set_variant: variant not available for this matrix");
+      if (!band_ok(s))
+        return fail(s, DETAG_ERR_UNSUPPORTED,
+                    "detag_set_variant: ring variant needs a circulant matrix, n a multiple of 32, n >= 64, K*bandwidth <= 16");
+      break;
     default:
       return fail(s, DETAG_ERR_ARG, "detag_set_variant: unknown variant");
   }

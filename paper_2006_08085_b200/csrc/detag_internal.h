@@ -61,6 +61,8 @@ int launch_step_csr(const StepParams& p, int sm_count, cudaStream_t stream);
 bool dense_variant_available(int n);  // n <= kMaxDenseWorkers and the driver offers tensor-map encoding
 int launch_step_dense(const StepParams& p, int sm_count, cudaStream_t stream);  // register-tiled, 32 < n <= 64
 int launch_step_mma(StepParams p, int sm_count, cudaStream_t stream);           // FP64 tensor path, n <= 32
+bool band_variant_available(int n, int half_band);  // circulant band kernel: n % 32 == 0, n >= 64, half-band <= 16
+int launch_step_band(StepParams p, const double* band, int sm_count, cudaStream_t stream);
 int launch_consensus_error(const StepParams& p, double* partials, double* result, int sm_count, cudaStream_t stream);
 
 }  // namespace detag
@@ -73,6 +75,9 @@ struct detag_state {
   std::vector<int32_t> row_ptr, col_idx;
   std::vector<double> vals;
   std::vector<double> poly;  // P_K(M) when n <= kMaxDenseWorkers
+  bool circulant = false;    // every row of M is the previous one shifted by one
+  int half_band = 0;         // of the circulant P_K(M): P[i][(i+delta) mod n] = 0 for |delta| > half_band
+  double band[33] = {0};     // p(delta) at index delta + 16, valid when circulant and half_band <= 16
   int variant_forced = DETAG_VARIANT_AUTO;
 
   bool bound = false;

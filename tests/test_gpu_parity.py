@@ -180,6 +180,31 @@ def test_noise_matches_the_counter_based_definition():
                 assert np.abs(err).max() < 6e-6 and np.sqrt((err ** 2).mean()) < 1e-6, (v, t, np.abs(err).max())
 
 
+@pytest.mark.parametrize("n,d,K,kind", [(64, 130, 16, "ring"), (96, 67, 5, "ring"), (64, 200, 4, "directed"),
+                                         (128, 64, 8, "two_hop"), (256, 129, 16, "slack")])
+def test_circulant_band_variant(n, d, K, kind):
+    """Circulant matrices take the banded-polynomial kernel: symmetric ring, a NON-symmetric circulant (fixes the
+    sign of the band offset), a two-hop circulant (bandwidth 2), and a slack ring."""
+    rng = np.random.default_rng(n + d)
+    if kind == "ring":
+        m = inputs.metropolis_weights(inputs.ring_graph(n))
+    elif kind == "slack":
+        m = inputs.slack_matrix(inputs.metropolis_weights(inputs.ring_graph(n)), 0.1)
+    elif kind == "directed":
+        m = inputs.directed_cycle_blend(n, 0.45, 0.35)
+    else:
+        dense = np.zeros((n, n))
+        for i in range(n):
+            for off, w in ((0, 0.4), (1, 0.2), (-1, 0.2), (2, 0.1), (-2, 0.1)):
+                dense[i, (i + off) % n] += w
+        m = inputs.csr_from_dense(dense)
+    assert B.DETAG_VARIANT_RING in _variants_for(m, K)
+    a, c = _random_objective(rng, n, d, scale=0.1)
+    x0 = rng.standard_normal((n, d)).astype(np.float32)
+    _check_one_step(m, K, 0.3, 0.02, a, c, x0, 0.1, 5, variants=[B.DETAG_VARIANT_RING])
+    _check_trajectory(m, K, 0.3, 0.02, a, c, x0, 0.1, 5, steps=5, variants=[B.DETAG_VARIANT_RING])
+
+
 def test_misuse_is_reported_not_faulted():
     import torch
 
