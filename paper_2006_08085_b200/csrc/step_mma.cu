@@ -80,6 +80,22 @@ __device__ __forceinline__ bool bar_wait(uint64_t* bar, unsigned parity) {
   return false;
 }
 
+// Monotonic progress counter in shared memory (release/acquire at CTA scope), bounded wait.
+__device__ __forceinline__ void count_publish(unsigned* counter, unsigned value) {
+  asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(s_addr(counter)), "r"(value) : "memory");
+}
+
+__device__ __forceinline__ bool count_wait(const unsigned* counter, unsigned at_least) {
+  const uint32_t addr = s_addr(counter);
+  for (unsigned spin = 0; spin < kMmaSpinLimit; ++spin) {
+    unsigned v;
+    asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    if (v >= at_least) return true;
+    __nanosleep(100);
+  }
+  return false;
+}
+
 __device__ __forceinline__ void bar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_addr(bar)) : "memory");
 }
@@ -121,6 +137,7 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
   uint64_t* empty = full + kMmaStages;
   uint64_t* out_ready = empty + kMmaStages;      // [group]: the group's 8 warps have written their outputs
   uint64_t* out_free = out_ready + kWarpGroups;  // [group]: the stores have finished reading the tile
+  unsigned* seen = reinterpret_cast<unsigned*>(out_free + kWarpGroups);  // [group]: 1 + last slab index whose data it saw
   if ((s_addr(smem_raw) & 127u) != 0) {
     if (threadIdx.x == 0) atomicExch(p.status, 2);
     return;
@@ -135,6 +152,7 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
     frag[e] = (i < n && j < n) ? p.poly[static_cast<size_t>(i) * n + j] : 0.0;
   }
   if (tid == 0) {
+    for (int g = 0; g < kWarpGroups; ++g) seen[g] = 0;
     for (int s = 0; s < kMmaStages; ++s) {
       bar_init(&full[s], 1);
       bar_init(&empty[s], kGroupWarps);
@@ -224,7 +242,13 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
     const int s = static_cast<int>(k % kMmaStages);
     bool ok = true;
     if (lane == 0) {
-      ok = bar_wait(&full[s], (k / kMmaStages) & 1);
+      // The stage last held slab k - kMmaStages, which belongs to the other group when the stage count is odd.
+      // A parity wait must not start before that phase has completed (it could not tell the two apart), and
+      // it costs nothing to make sure: this slab cannot have been loaded before that one was consumed.
+      if (kMmaStages % kWarpGroups != 0 && k >= kMmaStages)
+        ok = count_wait(&seen[(k - kMmaStages) % kWarpGroups], static_cast<unsigned>(k - kMmaStages + 1));
+      if (ok) ok = bar_wait(&full[s], (k / kMmaStages) & 1);
+      if (ok && tile == 0) count_publish(&seen[group], static_cast<unsigned>(k + 1));
       if (ok && use > 0) ok = bar_wait(&out_free[group], (use - 1) & 1);  // previous tile of this group stored
     }
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
