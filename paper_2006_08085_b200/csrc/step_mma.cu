@@ -264,14 +264,24 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
     const long long j0 = slab * kS;
 
     if (j0 + cl < p.d) {
+      // The two contractions are arranged so that the element-wise tail needs a single float64 addition:
+      //   cx accumulates P (x - alpha y) = x~ - alpha y~ = x'      (linearity of AG_K; Algorithm 2's model update)
+      //   cy starts at -g and accumulates P y, ending as y~ - g    (so the fold is y' = cy + g')
+      // Scalar float64 operations share the FP64 tensor pipe with the MMAs; every one issued from the tail
+      // queues behind other warps' MMAs, so as many as possible are done here, where this warp holds the pipe.
       double cy[4][2], cx[4][2];
 #pragma unroll
-      for (int t = 0; t < 4; ++t) cy[t][0] = cy[t][1] = cx[t][0] = cx[t][1] = 0.0;
+      for (int t = 0; t < 4; ++t) {
+        const float2 gv = *reinterpret_cast<const float2*>(sg + (4 * r + t) * kPitchE + cl + 2 * kq);
+        cy[t][0] = static_cast<double>(-gv.x);
+        cy[t][1] = static_cast<double>(-gv.y);
+        cx[t][0] = cx[t][1] = 0.0;
+      }
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         const int src = (4 * ks + kq) * kPitchXY + cl + r;
         const double by = static_cast<double>(sy[src]);
-        const double bx = static_cast<double>(sx[src]);
+        const double bx = fma(-alpha, by, static_cast<double>(sx[src]));
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
           const double a = frag[(t * 8 + ks) * 32 + lane];
@@ -295,24 +305,15 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
       for (int t = 0; t < 4; ++t) {
         const int row = 4 * r + t;
         const int eoff = row * kPitchE + cl + 2 * kq;
-        const float2 gv = *reinterpret_cast<const float2*>(sg + eoff);
         const float2 av = *reinterpret_cast<const float2*>(sa + eoff);
         const float2 cv = *reinterpret_cast<const float2*>(sc + eoff);
         float2 xo, yo, go;
-        {
-          const float x_new = static_cast<float>(fma(-alpha, cy[t][0], cx[t][0]));
-          const float g_new = fmaf(av.x, x_new - cv.x, sigma * xi[0][t]);
-          xo.x = x_new;
-          go.x = g_new;
-          yo.x = static_cast<float>(cy[t][0] + (static_cast<double>(g_new) - static_cast<double>(gv.x)));
-        }
-        {
-          const float x_new = static_cast<float>(fma(-alpha, cy[t][1], cx[t][1]));
-          const float g_new = fmaf(av.y, x_new - cv.y, sigma * xi[1][t]);
-          xo.y = x_new;
-          go.y = g_new;
-          yo.y = static_cast<float>(cy[t][1] + (static_cast<double>(g_new) - static_cast<double>(gv.y)));
-        }
+        xo.x = static_cast<float>(cx[t][0]);                           // x' (float64 accumulator, rounded once)
+        xo.y = static_cast<float>(cx[t][1]);
+        go.x = fmaf(av.x, xo.x - cv.x, sigma * xi[0][t]);              // stochastic gradient at the new model
+        go.y = fmaf(av.y, xo.y - cv.y, sigma * xi[1][t]);
+        yo.x = static_cast<float>(cy[t][0] + static_cast<double>(go.x));  // fold: (y~ - g) + g', g' as stored
+        yo.y = static_cast<float>(cy[t][1] + static_cast<double>(go.y));
         const int ooff = row * kS + cl + 2 * kq;
         *reinterpret_cast<float2*>(ob + ooff) = xo;
         *reinterpret_cast<float2*>(ob + kN * kS + ooff) = yo;
@@ -334,11 +335,13 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
         }
         if (p.y_obs != nullptr && row < n) {  // optional observer: the gossiped tracker, stored directly
           const long long off = static_cast<long long>(row) * p.ld + j;
+          const float2 gv = *reinterpret_cast<const float2*>(sg + eoff);
           if (j + 1 < p.d) {
             *reinterpret_cast<float2*>(p.y_obs + off) =
-                make_float2(static_cast<float>(cy[t][0]), static_cast<float>(cy[t][1]));
+                make_float2(static_cast<float>(cy[t][0] + static_cast<double>(gv.x)),
+                            static_cast<float>(cy[t][1] + static_cast<double>(gv.y)));
           } else if (j < p.d) {
-            p.y_obs[off] = static_cast<float>(cy[t][0]);
+            p.y_obs[off] = static_cast<float>(cy[t][0] + static_cast<double>(gv.x));
           }
         }
       }
