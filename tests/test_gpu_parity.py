@@ -327,3 +327,38 @@ def test_cfg4_full_size_sampled_blocks():
 def test_cfg3_full_size_sampled_blocks():
     d = inputs.CONFIGS["cfg3"].d
     _full_size_sampled("cfg3", [(0, 128), (7_000_003, 96), (d - 128, 128)], steps=10)
+
+
+# ----------------------------------------------------------------------------- host-resident stepping
+@pytest.mark.parametrize("n,d,K,graph", [(16, 100_003, 4, "ring"), (64, 20_000, 3, "ring"), (9, 5_001, 2, "path")])
+def test_step_host_matches_device_resident_stepping(n, d, K, graph):
+    """detag_step_host (state in page-locked host memory, chunked through a device staging area) performs the
+    same arithmetic per coordinate as detag_step: bit-identical results, several chunks and a ragged last one."""
+    import torch
+
+    rng = np.random.default_rng(n + d)
+    adj = inputs.ring_graph(n) if graph == "ring" else inputs.path_graph(n)
+    m = inputs.metropolis_weights(adj)
+    eta = orc.spectrum(m.to_dense()).eta
+    a, c = _random_objective(rng, n, d)
+    x0 = rng.standard_normal((n, d)).astype(np.float32)
+    with Session(m, d, K, eta, 0.05, a, c, x0, 0.1, 21) as s:
+        s.init()
+        ld = s.ld
+        host = {k: torch.empty((n, ld), dtype=torch.float32).pin_memory() for k in ("x", "y", "g", "a", "c")}
+        for k in host:
+            host[k].copy_(getattr(s, k))
+        torch.cuda.synchronize()
+        chunk = 128 * 64  # 8192 coordinates per chunk: d spans many chunks
+        nbytes = B.detag_host_staging_bytes(s.state, chunk)
+        staging = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda:0")
+        sptr = staging.data_ptr() + (-staging.data_ptr()) % 256
+        for step in range(3):
+            B.detag_set_step(s.state, step)
+            B.detag_step_host(s.state, ld, host["x"], host["y"], host["g"], host["a"], host["c"], sptr, nbytes,
+                              s.stream())
+            B.detag_set_step(s.state, step)
+            s.step()
+            torch.cuda.synchronize()
+            for k in ("x", "y", "g"):
+                assert torch.equal(host[k][:, :d], getattr(s, k)[:, :d].cpu()), (k, step)
