@@ -33,14 +33,17 @@ BYTES_PER_WC = 32  # read x, y, g, a, c + write x, y, g, float32 each: the fused
 # DRAM traffic per worker-coordinate (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture on a
 # small case of the same kernel; traffic grows in proportion to n*d).  Keyed by the sha256 prefix of the kernel
 # source the capture was taken on: a changed kernel reports null until it is captured again.
-MEASURED_TRAFFIC = {"step_mma.cu": ("740c172a2504ad82", 31.23)}
+MEASURED_TRAFFIC = {
+    "step_mma.cu": ("1f9c10577c38a0a4", 31.29),   # cfg5 shape, d = 2,000,000: 1.2835 GB read + 0.7189 GB written / 64 M wc
+    "step_band.cu": ("2fac1dfc9e253737", 31.10),  # cfg4 shape, d = 200,000: 1.0244 GB read + 0.5681 GB written / 51.2 M wc
+}
 
 
 def measured_traffic_bytes(variant: str, n: int, wc: int):
     import hashlib
-    if variant != "dense" or n > 32:
+    name = {"dense": "step_mma.cu" if n <= 32 else None, "ring": "step_band.cu"}.get(variant)
+    if name is None:
         return None
-    name = "step_mma.cu"
     digest, per_wc = MEASURED_TRAFFIC[name]
     path = os.path.join(ROOT, "paper_2006_08085_b200", "csrc", name)
     try:
