@@ -44,7 +44,8 @@ constexpr int kHalo = 16;          // window rows on each side = largest support
 constexpr int kW = kR + 2 * kHalo; // window rows
 constexpr int kS = 64;             // coordinates per tile: 8 MMA tiles of 8, one per consumer warp of a group
 constexpr int kPitchXY = kS + 8;   // floats; 8 mod 32 -> the four window rows of a B fragment hit disjoint banks
-constexpr int kPitchE = kS + 4;    // floats; rows of g, a, c (read in the accumulator layout)
+constexpr int kPitchE = kS + 8;    // floats; rows of g, a, c: consecutive rows 8t + r of the accumulator layout
+                                   // land 8 banks apart, so those loads are conflict-free as well
 constexpr int kStageFloats = 2 * kW * kPitchXY + 3 * kR * kPitchE;
 constexpr int kStageBytes = kStageFloats * 4;
 constexpr int kStages = 2;
@@ -120,6 +121,22 @@ __device__ __forceinline__ bool peers_wait(const unsigned* counters, int count, 
   return false;
 }
 
+// Monotonic progress counter in this CTA's shared memory (release/acquire at CTA scope), bounded wait.
+__device__ __forceinline__ void count_publish(unsigned* counter, unsigned value) {
+  asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(s_addr(counter)), "r"(value) : "memory");
+}
+
+__device__ __forceinline__ bool count_wait(const unsigned* counter, unsigned at_least) {
+  const uint32_t addr = s_addr(counter);
+  for (unsigned spin = 0; spin < kSpinLimit; ++spin) {
+    unsigned v;
+    asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    if (v >= at_least) return true;
+    __nanosleep(100);
+  }
+  return false;
+}
+
 __device__ __forceinline__ void bar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_addr(bar)) : "memory");
 }
@@ -174,6 +191,7 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
   uint64_t* out_ready = empty + kStages;
   uint64_t* out_free = out_ready + kWarpGroups;
   unsigned* landed = reinterpret_cast<unsigned*>(out_free + kWarpGroups);  // [peer]: slabs whose window peer has loaded
+  unsigned* seen = landed + kMaxCluster;  // [group]: 1 + index of the last slab whose data the group has seen
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = p.n;
   const int row_blocks = n / kR;             // = cluster size
@@ -181,6 +199,7 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
   const bool aligned_ok = (s_addr(smem_raw) & 127u) == 0;
   if (tid == 0) {
     for (int q = 0; q < kMaxCluster; ++q) landed[q] = 0;
+    for (int g = 0; g < kWarpGroups; ++g) seen[g] = 0;
     for (int s = 0; s < kStages; ++s) {
       bar_init(&full[s], 1);
       bar_init(&empty[s], kGroupWarps + 1);  // the group's warps + the signalling thread
@@ -303,7 +322,12 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
     const int s = static_cast<int>(k % kStages);
     bool ok = true;
     if (lane == 0) {
-      ok = bar_wait(&full[s], (k / kStages) & 1);
+      // with an odd stage count the stage last served the other group: a parity wait must not start before
+      // that phase has completed (it could not tell the two apart); the counter says when it has
+      if (kStages % kWarpGroups != 0 && k >= kStages)
+        ok = count_wait(&seen[(k - kStages) % kWarpGroups], static_cast<unsigned>(k - kStages + 1));
+      if (ok) ok = bar_wait(&full[s], (k / kStages) & 1);
+      if (ok && mtile == 0) count_publish(&seen[group], static_cast<unsigned>(k + 1));
       if (ok && use > 0) ok = bar_wait(&out_free[group], (use - 1) & 1);
     }
     const long long slab = tile;
@@ -323,14 +347,21 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
     const long long j0 = slab * kS;
 
     if (j0 + cl < p.d) {
+      // cx accumulates P (x - alpha y) = x' and cy starts at -g, ending as y~ - g: the tail then needs a single
+      // float64 addition (scalar float64 work queues behind other warps' MMAs on the shared FP64 pipe)
       double cy[4][2], cx[4][2];
 #pragma unroll
-      for (int t = 0; t < 4; ++t) cy[t][0] = cy[t][1] = cx[t][0] = cx[t][1] = 0.0;
+      for (int t = 0; t < 4; ++t) {
+        const float2 gv = *reinterpret_cast<const float2*>(sg + (8 * t + r) * kPitchE + cl + 2 * kq);
+        cy[t][0] = static_cast<double>(-gv.x);
+        cy[t][1] = static_cast<double>(-gv.y);
+        cx[t][0] = cx[t][1] = 0.0;
+      }
 #pragma unroll
       for (int ws = 0; ws < kW / 4; ++ws) {  // window steps of four rows
         const int src = (4 * ws + kq) * kPitchXY + cl + r;
         const double by = static_cast<double>(sy[src]);
-        const double bx = static_cast<double>(sx[src]);
+        const double bx = fma(-alpha, by, static_cast<double>(sx[src]));
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
           const int u = ws - 2 * t;  // compile-time after unrolling: only the band's blocks are issued
@@ -359,16 +390,15 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
       for (int t = 0; t < 4; ++t) {
         const int orow = 8 * t + r;  // output row within the tile
         const int eoff = orow * kPitchE + cl + 2 * kq;
-        const float2 gv = *reinterpret_cast<const float2*>(sg + eoff);
         const float2 av = *reinterpret_cast<const float2*>(sa + eoff);
         const float2 cv = *reinterpret_cast<const float2*>(sc + eoff);
         float2 xo, yo, go;
-        xo.x = static_cast<float>(fma(-alpha, cy[t][0], cx[t][0]));  // x' = x~ - alpha y~ (Algorithm 2)
-        xo.y = static_cast<float>(fma(-alpha, cy[t][1], cx[t][1]));
-        go.x = fmaf(av.x, xo.x - cv.x, sigma * xi[0][t]);            // stochastic gradient at the new model
+        xo.x = static_cast<float>(cx[t][0]);                              // x' (Algorithm 2's model update)
+        xo.y = static_cast<float>(cx[t][1]);
+        go.x = fmaf(av.x, xo.x - cv.x, sigma * xi[0][t]);                 // stochastic gradient at the new model
         go.y = fmaf(av.y, xo.y - cv.y, sigma * xi[1][t]);
-        yo.x = static_cast<float>(cy[t][0] + (static_cast<double>(go.x) - static_cast<double>(gv.x)));  // fold
-        yo.y = static_cast<float>(cy[t][1] + (static_cast<double>(go.y) - static_cast<double>(gv.y)));
+        yo.x = static_cast<float>(cy[t][0] + static_cast<double>(go.x));  // fold: (y~ - g) + g', g' as stored
+        yo.y = static_cast<float>(cy[t][1] + static_cast<double>(go.y));
         const int ooff = orow * kS + cl + 2 * kq;
         *reinterpret_cast<float2*>(ob + ooff) = xo;
         *reinterpret_cast<float2*>(ob + kR * kS + ooff) = yo;
@@ -387,11 +417,13 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
           }
         }
         if (p.y_obs != nullptr) {  // optional observer: the gossiped tracker, stored directly
+          const float2 gv = *reinterpret_cast<const float2*>(sg + eoff);
           if (j + 1 < p.d) {
             *reinterpret_cast<float2*>(p.y_obs + off) =
-                make_float2(static_cast<float>(cy[t][0]), static_cast<float>(cy[t][1]));
+                make_float2(static_cast<float>(cy[t][0] + static_cast<double>(gv.x)),
+                            static_cast<float>(cy[t][1] + static_cast<double>(gv.y)));
           } else if (j < p.d) {
-            p.y_obs[off] = static_cast<float>(cy[t][0]);
+            p.y_obs[off] = static_cast<float>(cy[t][0] + static_cast<double>(gv.x));
           }
         }
       }
