@@ -184,6 +184,61 @@ def folded_tracker(s: State) -> np.ndarray:
     return fold(s.y, s.g_new, s.g_old)
 
 
+# --------------------------------------------------------------------------------------
+# Algorithm 2 with the timing it prints: the gradient of phase k is queried at the phase-start point
+# --------------------------------------------------------------------------------------
+class PhaseState(NamedTuple):
+    """State at the start of phase k of Algorithm 2 read literally."""
+    x: np.ndarray  # x_k
+    y: np.ndarray  # tracker y_k as the algorithm holds it (the fold of phase k-1 already applied)
+    g_prev: np.ndarray  # gradient buffer g_(k-1)
+    t: int  # number of completed phases
+
+
+def init_phase_state(p: Problem, x0: np.ndarray) -> PhaseState:
+    """Same start as ``init_state``: y_0 = g_(-1) = stochastic gradient at x_0 (noise index 0)."""
+    x = np.array(x0, dtype=np.float64, copy=True)
+    g = stochastic_gradient(p, x, 0)
+    return PhaseState(x, g.copy(), g, 0)
+
+
+def phase_as_printed(p: Problem, s: PhaseState) -> PhaseState:
+    """One phase of Algorithm 2 in the order the algorithm box prints it.
+
+    While the K gossip rounds run on the model replica and on the tracker, the gradient oracle is
+    queried at the phase-start point x_k (the box's "compute stochastic gradient at point x_k");
+    at the end of the phase the model is updated with the gossiped tracker and only then is the
+    tracker folded with g_(k) - g_(k-1).  Compared with ``step`` the gradient that enters a fold
+    is one phase older.
+    """
+    g = stochastic_gradient(p, s.x, s.t + 1)
+    y_gossip = accelerated_gossip(s.y, p.row_ptr, p.col_idx, p.vals, p.K, p.eta)
+    x_tilde = accelerated_gossip(s.x, p.row_ptr, p.col_idx, p.vals, p.K, p.eta)
+    x = x_tilde - p.alpha * y_gossip
+    y = y_gossip + g - s.g_prev
+    return PhaseState(x, y, g, s.t + 1)
+
+
+def run_as_printed(p: Problem, x0: np.ndarray, phases: int, observe=None) -> PhaseState:
+    s = init_phase_state(p, x0)
+    if observe is not None:
+        observe(s)
+    for _ in range(phases):
+        s = phase_as_printed(p, s)
+        if observe is not None:
+            observe(s)
+    return s
+
+
+def phase_length(n: int, lam: float, varsigma0_sq: float, T: float, delta_L: float) -> int:
+    """Theorem 3's phase length R = max(1/2 ln n, 1/2 ln(varsigma_0^2 T / (Delta L))) / sqrt(1 - lambda),
+    rounded up to a whole number of gossip rounds (at least one)."""
+    terms = [0.5 * math.log(n)]
+    if varsigma0_sq > 0.0 and T > 0.0 and delta_L > 0.0:
+        terms.append(0.5 * math.log(varsigma0_sq * T / delta_L))
+    return max(1, math.ceil(max(terms) / math.sqrt(1.0 - lam)))
+
+
 def consensus_error(x: np.ndarray) -> float:
     """||X - Xbar 1^T||_F^2 = sum_j sum_i (x_ij - mean_i x_ij)^2."""
     x = np.asarray(x, dtype=np.float64)

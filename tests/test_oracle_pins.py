@@ -338,3 +338,91 @@ def test_parity_helper_is_the_same_cycle_cut_elsewhere():
     s1 = orc.step(p, s0)
     assert np.array_equal(s1.x, x1) and np.array_equal(s1.y, yg1) and np.array_equal(s1.g_new, g1)
     assert np.array_equal(orc.folded_tracker(s1), yf1)
+
+
+# ----------------------------------------------------------------------------- Algorithm 2 with its printed timing
+def _dense_polynomial(dense, K, eta):
+    """P_K by explicit matrix products (brute force, independent of the oracle's row-wise rounds)."""
+    prev = np.eye(dense.shape[0])
+    cur = prev.copy()
+    for _ in range(K):
+        prev, cur = cur, (1.0 + eta) * dense @ cur - eta * prev
+    return cur
+
+
+def test_printed_timing_matches_dense_matrix_recursion():
+    """x_{k+1} = P x_k - alpha P y_k, y_{k+1} = P y_k + g(x_k) - g(x_{k-1}) with P from brute-force matrix products."""
+    p, w = _small_problem(11, n=8, m=7, K=3, sigma=0.0, alpha=0.03)
+    P = _dense_polynomial(w.to_dense(), p.K, p.eta)
+    a, c = p.a.astype(np.float64), p.c.astype(np.float64)
+    x = np.random.default_rng(2).standard_normal((8, 7))
+    g_prev = a * (x - c)
+    y = g_prev.copy()
+    s = orc.init_phase_state(p, x)
+    for _ in range(5):
+        g = a * (x - c)  # at the phase-start point
+        x, y, g_prev = P @ x - p.alpha * (P @ y), P @ y + g - g_prev, g
+        s = orc.phase_as_printed(p, s)
+        assert np.allclose(s.x, x, atol=1e-12) and np.allclose(s.y, y, atol=1e-12)
+        assert np.allclose(s.g_prev, g_prev, atol=1e-12)
+
+
+def test_printed_timing_tracker_sum_and_stale_mean_descent():
+    """Proof of Theorem 3: mean tracker = mean of the previous phase's gradients; mean model descends along it."""
+    p, _ = _small_problem(12, sigma=0.2)
+    s = orc.init_phase_state(p, np.random.default_rng(3).standard_normal((8, 6)))
+    for _ in range(6):
+        assert np.allclose(s.y.sum(0), s.g_prev.sum(0), atol=1e-10)
+        nxt = orc.phase_as_printed(p, s)
+        assert np.allclose(nxt.x.mean(0), s.x.mean(0) - p.alpha * s.g_prev.mean(0), atol=1e-12)
+        # the gradient that entered this phase's fold was taken at the phase-start point, with this phase's noise
+        assert np.array_equal(nxt.g_prev, orc.stochastic_gradient(p, s.x, s.t + 1))
+        s = nxt
+
+
+def test_printed_timing_average_consensus_is_delayed_sgd():
+    """W = J/n, noise free: xbar_{k+1} = xbar_k - alpha mean_i a_i (x_{k-1,i} - c_i): gradient descent with delay one."""
+    n, m, alpha = 5, 4, 0.1
+    w = inputs.average_consensus_matrix(n)
+    rng = np.random.default_rng(5)
+    a = rng.uniform(0.5, 2.0, (n, m))
+    c = rng.standard_normal((n, m))
+    p = _problem(w, 1, 0.0, alpha, a, c, 0.0)
+    s = orc.init_phase_state(p, np.zeros((n, m)))
+    x_older = np.zeros(m)  # x_{-1} := x_0 (the initial buffer holds the gradient at x_0)
+    x_cur = np.zeros(m)
+    for _ in range(6):
+        s = orc.phase_as_printed(p, s)
+        x_older, x_cur = x_cur, x_cur - alpha * (a * (x_older[None, :] - c)).mean(0)
+        assert np.allclose(s.x, np.tile(x_cur, (n, 1)), atol=1e-12)
+
+
+def test_printed_timing_has_the_same_fixed_point():
+    p, _ = _small_problem(13, n=8, m=5, K=4, sigma=0.0, alpha=0.05)
+    s = orc.run_as_printed(p, np.zeros((8, 5)), 800)
+    a, c = p.a.astype(np.float64), p.c.astype(np.float64)
+    xstar = (a * c).sum(0) / a.sum(0)
+    assert np.allclose(s.x, np.tile(xstar, (8, 1)), atol=1e-9) and np.abs(s.y).max() < 1e-8
+
+
+def test_printed_timing_differs_from_the_fresh_gradient_step_only_by_the_gradient_point():
+    """Feeding the fresh-gradient step's fold a gradient taken at the old model reproduces the printed phase."""
+    p, _ = _small_problem(14, sigma=0.0)
+    x0 = np.random.default_rng(6).standard_normal((8, 6))
+    s = orc.init_phase_state(p, x0)
+    x_new, y_gossip = orc.gossip_and_update(p, s.x, s.y)
+    nxt = orc.phase_as_printed(p, s)
+    assert np.array_equal(nxt.x, x_new)
+    assert np.allclose(nxt.y, orc.fold(y_gossip, orc.gradient(s.x, p.a, p.c, 0.0, None), s.g_prev), atol=1e-13)
+
+
+def test_phase_length_of_theorem_3():
+    # sqrt(1 - lambda) = 1/2: R = ln(16) = 2.77 -> 3 rounds; the data-heterogeneity term takes over when it is larger
+    assert orc.phase_length(16, 0.75, 0.0, 0.0, 1.0) == 3
+    assert orc.phase_length(16, 0.75, 4.0, 1e6, 2.0) == math.ceil(math.log(2e6))  # = ceil(0.5 ln(2e6) / 0.5) = 15
+    assert orc.phase_length(2, 0.0, 0.0, 0.0, 1.0) == 1
+    # the 256-worker Metropolis ring: lambda = (1 + 2 cos(2 pi/256))/3, R = 0.5 ln 256 / sqrt(1 - lambda) = 195.6
+    lam = (1.0 + 2.0 * math.cos(2.0 * math.pi / 256)) / 3.0
+    assert orc.phase_length(256, lam, 0.0, 0.0, 1.0) == 196
+    # doubling the spectral gap's square root halves the phase
+    assert orc.phase_length(1 << 20, 1.0 - 1e-4, 0.0, 0.0, 1.0) == math.ceil(0.5 * math.log(1 << 20) / 1e-2)
