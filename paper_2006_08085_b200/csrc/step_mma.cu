@@ -22,7 +22,11 @@
 //             come from L2) and are not used.
 //   consumers 16 warps in two groups that take alternate slabs; a warp owns 8 coordinates of the slab:
 //             64 MMAs, then the element-wise tail (model update, Philox/Box-Muller noise, gradient,
-//             tracker fold), results written to the group's dense output tile in shared memory.
+//             tracker fold), results written to the group's dense output tile in shared memory.  The
+//             tail's inputs (a, c) are copied to registers after the MMAs and the stage is handed back
+//             to the producer before the tail starts: with three stages and two groups, a stage held
+//             through the tail leaves a single stage of loads in flight, which is too little to cover
+//             the HBM latency (measured: 5.27 -> 4.88 ms per step at n = 32, d = 25.6 M).
 //   storer    one thread writes each finished output tile (x', y', g': 32 rows x 256 bytes) with three
 //             TMA tile stores.  Row-contiguous 256-byte writes matter: storing straight from the
 //             accumulator layout (32-byte pieces of 8 rows per instruction) halves the HBM throughput.
@@ -249,7 +253,6 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
         ok = count_wait(&seen[(k - kMmaStages) % kWarpGroups], static_cast<unsigned>(k - kMmaStages + 1));
       if (ok) ok = bar_wait(&full[s], (k / kMmaStages) & 1);
       if (ok && tile == 0) count_publish(&seen[group], static_cast<unsigned>(k + 1));
-      if (ok && use > 0) ok = bar_wait(&out_free[group], (use - 1) & 1);  // previous tile of this group stored
     }
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     if (!ok) {
@@ -263,13 +266,15 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
     const float* sc = sa + kN * kPitchE;
     const long long j0 = slab * kS;
 
-    if (j0 + cl < p.d) {
+    const bool active = j0 + cl < p.d;  // a tile wholly beyond column d computes nothing but keeps the protocol
+    double cy[4][2], cx[4][2];
+    float2 av4[4], cv4[4], gv4[4];
+    if (active) {
       // The two contractions are arranged so that the element-wise tail needs a single float64 addition:
       //   cx accumulates P (x - alpha y) = x~ - alpha y~ = x'      (linearity of AG_K; Algorithm 2's model update)
       //   cy starts at -g and accumulates P y, ending as y~ - g    (so the fold is y' = cy + g')
       // Scalar float64 operations share the FP64 tensor pipe with the MMAs; every one issued from the tail
       // queues behind other warps' MMAs, so as many as possible are done here, where this warp holds the pipe.
-      double cy[4][2], cx[4][2];
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const float2 gv = *reinterpret_cast<const float2*>(sg + (4 * r + t) * kPitchE + cl + 2 * kq);
@@ -289,6 +294,26 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
           dmma(cx[t], a, bx);
         }
       }
+      // the tail's inputs move to registers so that the stage can be refilled while the tail runs
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int eoff = (4 * r + t) * kPitchE + cl + 2 * kq;
+        av4[t] = *reinterpret_cast<const float2*>(sa + eoff);
+        cv4[t] = *reinterpret_cast<const float2*>(sc + eoff);
+        if (p.y_obs != nullptr) gv4[t] = *reinterpret_cast<const float2*>(sg + eoff);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) {
+      bar_arrive(&empty[s]);                                                       // stage no longer read by this warp
+      if (use > 0) ok = bar_wait(&out_free[group], (use - 1) & 1);                 // previous tile of this group stored
+    }
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    if (!ok) {
+      if (lane == 0) atomicExch(p.status, 1);
+      return;
+    }
+    if (active) {
       // element-wise tail: workers 4r..4r+3 (index t), coordinates j, j+1
       const long long j = j0 + cl + 2 * kq;
       float xi[2][4];
@@ -304,9 +329,7 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const int row = 4 * r + t;
-        const int eoff = row * kPitchE + cl + 2 * kq;
-        const float2 av = *reinterpret_cast<const float2*>(sa + eoff);
-        const float2 cv = *reinterpret_cast<const float2*>(sc + eoff);
+        const float2 av = av4[t], cv = cv4[t];
         float2 xo, yo, go;
         xo.x = static_cast<float>(cx[t][0]);                           // x' (float64 accumulator, rounded once)
         xo.y = static_cast<float>(cx[t][1]);
@@ -335,7 +358,7 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
         }
         if (p.y_obs != nullptr && row < n) {  // optional observer: the gossiped tracker, stored directly
           const long long off = static_cast<long long>(row) * p.ld + j;
-          const float2 gv = *reinterpret_cast<const float2*>(sg + eoff);
+          const float2 gv = gv4[t];
           if (j + 1 < p.d) {
             *reinterpret_cast<float2*>(p.y_obs + off) =
                 make_float2(static_cast<float>(cy[t][0] + static_cast<double>(gv.x)),
@@ -346,13 +369,10 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
         }
       }
     }
-    // outputs visible to the TMA store, input stage no longer read by this warp
+    // outputs visible to the TMA store
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
-    if (lane == 0) {
-      bar_arrive(&out_ready[group]);
-      bar_arrive(&empty[s]);
-    }
+    if (lane == 0) bar_arrive(&out_ready[group]);
   }
 }
 
