@@ -62,6 +62,12 @@ enum {
   DETAG_VARIANT_RING = 3   /* banded circulant polynomial P_K(M): circulant M (rings), n % 32 == 0, n >= 64, K*bandwidth <= 16 */
 };
 
+/* The point at which a step queries the stochastic gradient oracle. */
+enum {
+  DETAG_GRADIENT_AT_NEW_MODEL = 0,   /* at x', the model the step produces (default; the step listing above) */
+  DETAG_GRADIENT_AT_PHASE_START = 1  /* at x, the model the step started from: Algorithm 2 as printed */
+};
+
 /*
  * Spectrum of a symmetric gossip matrix and the accelerated-gossip momentum.
  * Paper: Section "Protocol Layer" (lambda = max(|lambda_2|, |lambda_n|)) and Algorithm 3
@@ -120,6 +126,26 @@ int detag_set_noise(detag_state* s, double sigma, uint64_t seed, int64_t coord_o
 int detag_set_variant(detag_state* s, int variant);
 /* The variant the next detag_step will run (never AUTO). */
 int detag_get_variant(const detag_state* s, int* variant);
+
+/*
+ * Where the stochastic gradient of a step is evaluated (DETAG_GRADIENT_AT_*).
+ * Algorithm 2 as printed queries the oracle during the K gossip rounds of a phase, at the point x_k
+ * the phase started from, and folds g_(k) - g_(k-1) into the tracker at the end of the phase; its
+ * gradients are therefore one phase older than with the default, which evaluates at the new model:
+ *     g'  = a o (x - c) + sigma * xi     (x = the model before this step's update)
+ * Everything else in the step listing at the top is unchanged, and so is detag_init.  Errors: ARG.
+ */
+int detag_set_gradient_point(detag_state* s, int where);
+int detag_get_gradient_point(const detag_state* s, int* where);
+
+/*
+ * Phase length of Theorem 3: R = max(1/2 ln n, 1/2 ln(varsigma0_sq * T / delta_L)) / sqrt(1 - lambda),
+ * rounded up to a whole number of gossip rounds, at least 1.  lambda as returned by detag_spectral,
+ * varsigma0_sq the bound on the gradient dissimilarity at the origin (Section "Setting"), T the
+ * number of iterations, delta_L the product Delta * L; the second term is left out when any of
+ * varsigma0_sq, T, delta_L is not positive.  Host only.  Errors: ARG (n < 1, lambda outside [0, 1), null R).
+ */
+int detag_phase_length(int n, double lambda, double varsigma0_sq, double T, double delta_L, int* R);
 
 /*
  * Initial state of Algorithm 2 as the task fixes it: g = stochastic gradient at the bound x

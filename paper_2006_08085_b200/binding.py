@@ -32,6 +32,9 @@ DETAG_VARIANT_CSR = 1
 DETAG_VARIANT_DENSE = 2
 DETAG_VARIANT_RING = 3
 
+DETAG_GRADIENT_AT_NEW_MODEL = 0
+DETAG_GRADIENT_AT_PHASE_START = 1
+
 _ERR_NAMES = {
     -1: "DETAG_ERR_ARG", -2: "DETAG_ERR_CSR", -3: "DETAG_ERR_NOT_STOCHASTIC", -4: "DETAG_ERR_NOT_SYMMETRIC",
     -5: "DETAG_ERR_UNSUPPORTED", -6: "DETAG_ERR_UNBOUND", -7: "DETAG_ERR_CUDA", -8: "DETAG_ERR_TIMEOUT",
@@ -52,6 +55,10 @@ SIGNATURES = {
     "detag_set_noise": (ctypes.c_int, [_P, ctypes.c_double, ctypes.c_uint64, ctypes.c_int64]),
     "detag_set_variant": (ctypes.c_int, [_P, ctypes.c_int]),
     "detag_get_variant": (ctypes.c_int, [_P, ctypes.POINTER(ctypes.c_int)]),
+    "detag_set_gradient_point": (ctypes.c_int, [_P, ctypes.c_int]),
+    "detag_get_gradient_point": (ctypes.c_int, [_P, ctypes.POINTER(ctypes.c_int)]),
+    "detag_phase_length": (ctypes.c_int, [ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                          ctypes.c_double, ctypes.POINTER(ctypes.c_int)]),
     "detag_init": (ctypes.c_int, [_P, _P]),
     "detag_step": (ctypes.c_int, [_P, _P]),
     "detag_step_host": (ctypes.c_int, [_P, ctypes.c_int64, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P]),
@@ -166,6 +173,24 @@ def detag_set_variant(state, variant: int) -> None:
 def detag_get_variant(state) -> int:
     out = ctypes.c_int(0)
     _check(lib().detag_get_variant(state, ctypes.byref(out)), "detag_get_variant", state)
+    return int(out.value)
+
+
+def detag_set_gradient_point(state, where: int) -> None:
+    _check(lib().detag_set_gradient_point(state, int(where)), "detag_set_gradient_point", state)
+
+
+def detag_get_gradient_point(state) -> int:
+    out = ctypes.c_int(0)
+    _check(lib().detag_get_gradient_point(state, ctypes.byref(out)), "detag_get_gradient_point", state)
+    return int(out.value)
+
+
+def detag_phase_length(n: int, lam: float, varsigma0_sq: float = 0.0, T: float = 0.0, delta_L: float = 1.0) -> int:
+    """Theorem 3's phase length (gossip rounds per phase), host only."""
+    out = ctypes.c_int(0)
+    _check(lib().detag_phase_length(int(n), float(lam), float(varsigma0_sq), float(T), float(delta_L),
+                                    ctypes.byref(out)), "detag_phase_length")
     return int(out.value)
 
 

@@ -140,6 +140,7 @@ StepParams make_params(const detag_state* s) {
   p.seed_lo = static_cast<uint32_t>(s->seed & 0xffffffffu);
   p.seed_hi = static_cast<uint32_t>(s->seed >> 32);
   p.status = s->d_status;
+  p.grad_at_start = s->gradient_point == DETAG_GRADIENT_AT_PHASE_START ? 1 : 0;
   return p;
 }
 
@@ -336,6 +337,32 @@ int detag_set_variant(detag_state* s, int variant) {
 int detag_get_variant(const detag_state* s, int* variant) {
   if (!s || !variant) return DETAG_ERR_ARG;
   *variant = resolve_variant(s);
+  return DETAG_OK;
+}
+
+int detag_set_gradient_point(detag_state* s, int where) {
+  if (!s) return DETAG_ERR_ARG;
+  if (where != DETAG_GRADIENT_AT_NEW_MODEL && where != DETAG_GRADIENT_AT_PHASE_START)
+    return fail(s, DETAG_ERR_ARG, "detag_set_gradient_point: unknown value");
+  s->gradient_point = where;
+  return DETAG_OK;
+}
+
+int detag_get_gradient_point(const detag_state* s, int* where) {
+  if (!s || !where) return DETAG_ERR_ARG;
+  *where = s->gradient_point;
+  return DETAG_OK;
+}
+
+int detag_phase_length(int n, double lambda, double varsigma0_sq, double T, double delta_L, int* R) {
+  if (!R || n < 1 || !(lambda >= 0.0) || !(lambda < 1.0)) return DETAG_ERR_ARG;
+  double num = 0.5 * std::log(static_cast<double>(n));
+  if (varsigma0_sq > 0.0 && T > 0.0 && delta_L > 0.0) {
+    const double second = 0.5 * std::log(varsigma0_sq * T / delta_L);
+    if (second > num) num = second;
+  }
+  const double r = std::ceil(num / std::sqrt(1.0 - lambda));
+  *R = r < 1.0 ? 1 : (r > 2147483647.0 ? 2147483647 : static_cast<int>(r));
   return DETAG_OK;
 }
 

@@ -44,6 +44,7 @@ struct StepParams {
   double sigma;
   uint32_t seed_lo, seed_hi;
   uint32_t t_noise;  // step index that enters the noise counter
+  int grad_at_start;  // nonzero: the gradient is taken at the model the step started from (Algorithm 2 as printed)
   int* status;
 };
 
@@ -79,6 +80,7 @@ struct detag_state {
   int half_band = 0;         // of the circulant P_K(M): P[i][(i+delta) mod n] = 0 for |delta| > half_band
   double band[33] = {0};     // p(delta) at index delta + 16, valid when circulant and half_band <= 16
   int variant_forced = DETAG_VARIANT_AUTO;
+  int gradient_point = DETAG_GRADIENT_AT_NEW_MODEL;
 
   bool bound = false;
   long long ld = 0;

@@ -395,8 +395,13 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
         float2 xo, yo, go;
         xo.x = static_cast<float>(cx[t][0]);                              // x' (Algorithm 2's model update)
         xo.y = static_cast<float>(cx[t][1]);
-        go.x = fmaf(av.x, xo.x - cv.x, sigma * xi[0][t]);                 // stochastic gradient at the new model
-        go.y = fmaf(av.y, xo.y - cv.y, sigma * xi[1][t]);
+        float2 x_at = xo;  // gradient point: the new model, or (Algorithm 2 as printed) the model before this step,
+        if (p.grad_at_start) {  // which sits in the window: output row orow is window row orow + kHalo
+          const float* xw = sx + (orow + kHalo) * kPitchXY + cl + 2 * kq;
+          x_at = make_float2(xw[0], xw[1]);
+        }
+        go.x = fmaf(av.x, x_at.x - cv.x, sigma * xi[0][t]);               // stochastic gradient
+        go.y = fmaf(av.y, x_at.y - cv.y, sigma * xi[1][t]);
         yo.x = static_cast<float>(cy[t][0] + static_cast<double>(go.x));  // fold: (y~ - g) + g', g' as stored
         yo.y = static_cast<float>(cy[t][1] + static_cast<double>(go.y));
         const int ooff = orow * kS + cl + 2 * kq;

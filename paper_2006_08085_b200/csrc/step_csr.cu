@@ -105,7 +105,10 @@ __global__ void __launch_bounds__(kCsrThreads) step_csr_kernel(const StepParams 
           const long long off = static_cast<long long>(i) * p.ld + j;
           const double y_gossip = cy[i * S + col];
           const double x_new = cx[i * S + col] - alpha * y_gossip;
-          const double g_new = fma(static_cast<double>(p.a[off]), x_new - static_cast<double>(p.c[off]),
+          // gradient point: the new model, or (Algorithm 2 as printed) the model this step started from,
+          // which is still in global memory because this thread overwrites it only below
+          const double x_at = p.grad_at_start ? static_cast<double>(p.x[off]) : x_new;
+          const double g_new = fma(static_cast<double>(p.a[off]), x_at - static_cast<double>(p.c[off]),
                                    sigma * static_cast<double>(xi[w]));
           const float g_new_f = static_cast<float>(g_new);
           const double y_new = y_gossip + (static_cast<double>(g_new_f) - static_cast<double>(p.g[off]));

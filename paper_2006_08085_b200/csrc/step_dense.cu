@@ -244,9 +244,12 @@ step_dense_kernel(const StepParams p, const __grid_constant__ DenseMaps maps) {
       const float2 cv = *reinterpret_cast<const float2*>(sc + row * S + 2 * cg);
       const float2 gv = *reinterpret_cast<const float2*>(sg + row * S + 2 * cg);
       float2 xo, yo, go, yg;
+      // gradient point: the new model, or (Algorithm 2 as printed) the staged model this step started from
+      float2 x_at = make_float2(0.f, 0.f);
+      if (p.grad_at_start) x_at = *reinterpret_cast<const float2*>(sx + row * S + 2 * cg);
       {
         const float x_new = accx[i][0] - static_cast<float>(alpha * accy[i][0]);
-        const float g_new = fmaf(av.x, x_new - cv.x, sigma * xi[0][i]);
+        const float g_new = fmaf(av.x, (p.grad_at_start ? x_at.x : x_new) - cv.x, sigma * xi[0][i]);
         xo.x = x_new;
         go.x = g_new;
         yo.x = static_cast<float>(accy[i][0] + (static_cast<double>(g_new) - static_cast<double>(gv.x)));
@@ -254,7 +257,7 @@ step_dense_kernel(const StepParams p, const __grid_constant__ DenseMaps maps) {
       }
       {
         const float x_new = accx[i][1] - static_cast<float>(alpha * accy[i][1]);
-        const float g_new = fmaf(av.y, x_new - cv.y, sigma * xi[1][i]);
+        const float g_new = fmaf(av.y, (p.grad_at_start ? x_at.y : x_new) - cv.y, sigma * xi[1][i]);
         xo.y = x_new;
         go.y = g_new;
         yo.y = static_cast<float>(accy[i][1] + (static_cast<double>(g_new) - static_cast<double>(gv.y)));

@@ -129,6 +129,8 @@ __device__ __forceinline__ void dmma(double (&c)[2], double a, double b) {
                : "d"(a), "d"(b));
 }
 
+// kAtStart: the gradient is taken at the model the step started from (Algorithm 2 as printed) instead of the new one.
+template <bool kAtStart>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
   // No static shared memory in this kernel: the dynamic array starts at the CTA's shared window, whose
@@ -266,15 +268,15 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
     const float* sc = sa + kN * kPitchE;
     const long long j0 = slab * kS;
 
-    const bool active = j0 + cl < p.d;  // a tile wholly beyond column d computes nothing but keeps the protocol
-    double cy[4][2], cx[4][2];
-    float2 av4[4], cv4[4], gv4[4];
-    if (active) {
+    // A tile wholly beyond column d computes nothing but keeps the barrier protocol.
+    bool released = false, out_ok = true;
+    if (j0 + cl < p.d) {
       // The two contractions are arranged so that the element-wise tail needs a single float64 addition:
       //   cx accumulates P (x - alpha y) = x~ - alpha y~ = x'      (linearity of AG_K; Algorithm 2's model update)
       //   cy starts at -g and accumulates P y, ending as y~ - g    (so the fold is y' = cy + g')
       // Scalar float64 operations share the FP64 tensor pipe with the MMAs; every one issued from the tail
       // queues behind other warps' MMAs, so as many as possible are done here, where this warp holds the pipe.
+      double cy[4][2], cx[4][2];
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const float2 gv = *reinterpret_cast<const float2*>(sg + (4 * r + t) * kPitchE + cl + 2 * kq);
@@ -295,6 +297,7 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
         }
       }
       // the tail's inputs move to registers so that the stage can be refilled while the tail runs
+      float2 av4[4], cv4[4], gv4[4];
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const int eoff = (4 * r + t) * kPitchE + cl + 2 * kq;
@@ -302,18 +305,17 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
         cv4[t] = *reinterpret_cast<const float2*>(sc + eoff);
         if (p.y_obs != nullptr) gv4[t] = *reinterpret_cast<const float2*>(sg + eoff);
       }
-    }
-    __syncwarp();
-    if (lane == 0) {
-      bar_arrive(&empty[s]);                                                       // stage no longer read by this warp
-      if (use > 0) ok = bar_wait(&out_free[group], (use - 1) & 1);                 // previous tile of this group stored
-    }
-    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-    if (!ok) {
-      if (lane == 0) atomicExch(p.status, 1);
-      return;
-    }
-    if (active) {
+      __syncwarp();
+      if (lane == 0) {
+        bar_arrive(&empty[s]);
+        released = true;
+        if (use > 0 && !bar_wait(&out_free[group], (use - 1) & 1)) out_ok = false;  // previous tile stored
+      }
+      out_ok = __shfl_sync(0xffffffffu, out_ok ? 1 : 0, 0) != 0;
+      if (!out_ok) {
+        if (lane == 0) atomicExch(p.status, 1);
+        return;
+      }
       // element-wise tail: workers 4r..4r+3 (index t), coordinates j, j+1
       const long long j = j0 + cl + 2 * kq;
       float xi[2][4];
@@ -329,12 +331,21 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const int row = 4 * r + t;
-        const float2 av = av4[t], cv = cv4[t];
+        const int eoff = row * kPitchE + cl + 2 * kq;
+        const float2 av = av4[t];
+        const float2 cv = cv4[t];
         float2 xo, yo, go;
         xo.x = static_cast<float>(cx[t][0]);                           // x' (float64 accumulator, rounded once)
         xo.y = static_cast<float>(cx[t][1]);
-        go.x = fmaf(av.x, xo.x - cv.x, sigma * xi[0][t]);              // stochastic gradient at the new model
-        go.y = fmaf(av.y, xo.y - cv.y, sigma * xi[1][t]);
+        float2 x_at = xo;  // gradient point: the new model, or (Algorithm 2 as printed) the model before this step.
+        if (kAtStart && row < n) {
+          // The old model is still in global memory: this slab's stores are issued after all of its tails.
+          const long long off = static_cast<long long>(row) * p.ld + j;
+          x_at.x = j < p.d ? p.x[off] : 0.f;
+          x_at.y = j + 1 < p.d ? p.x[off + 1] : 0.f;
+        }
+        go.x = fmaf(av.x, x_at.x - cv.x, sigma * xi[0][t]);            // stochastic gradient
+        go.y = fmaf(av.y, x_at.y - cv.y, sigma * xi[1][t]);
         yo.x = static_cast<float>(cy[t][0] + static_cast<double>(go.x));  // fold: (y~ - g) + g', g' as stored
         yo.y = static_cast<float>(cy[t][1] + static_cast<double>(go.y));
         const int ooff = row * kS + cl + 2 * kq;
@@ -372,7 +383,13 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
     // outputs visible to the TMA store
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
-    if (lane == 0) bar_arrive(&out_ready[group]);
+    if (!(j0 + cl < p.d)) {  // idle tile
+      if (lane == 0 && use > 0 && !bar_wait(&out_free[group], (use - 1) & 1)) atomicExch(p.status, 1);
+    }
+    if (lane == 0) {
+      bar_arrive(&out_ready[group]);
+      if (!released) bar_arrive(&empty[s]);
+    }
   }
 }
 
@@ -391,12 +408,13 @@ int launch_step_mma(StepParams p, int sm_count, cudaStream_t stream) {
   if (d_tma == 0) maps.xs = maps.ys = maps.gs = maps.x;  // never used: every slab lies beyond column 0
   p.S = kS;
   p.num_slabs = (p.d + kS - 1) / kS;
-  cudaError_t e = cudaFuncSetAttribute(step_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  auto kernel = p.grad_at_start ? step_mma_kernel<true> : step_mma_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(kMmaSmemBytes));
   if (e != cudaSuccess) return static_cast<int>(e);
   const long long grid = p.num_slabs < sm_count ? p.num_slabs : sm_count;
   if (grid <= 0) return 0;
-  step_mma_kernel<<<static_cast<unsigned>(grid), kMmaThreads, kMmaSmemBytes, stream>>>(p, maps);
+  kernel<<<static_cast<unsigned>(grid), kMmaThreads, kMmaSmemBytes, stream>>>(p, maps);
   return static_cast<int>(cudaGetLastError());
 }
 

@@ -23,7 +23,8 @@ class Session:
 
     def __init__(self, m, d: int, K: int, eta: float, alpha: float, a=None, c=None, x0=None, sigma: float = 0.0,
                  seed: int = 0, coord_offset: int = 0, ld: Optional[int] = None, device: str = "cuda:0",
-                 observe_gossip: bool = False, variant: int = B.DETAG_VARIANT_AUTO):
+                 observe_gossip: bool = False, variant: int = B.DETAG_VARIANT_AUTO,
+                 gradient_point: int = B.DETAG_GRADIENT_AT_NEW_MODEL):
         import torch
 
         if not torch.cuda.is_available():
@@ -54,6 +55,8 @@ class Session:
             B.detag_observe_gossiped_tracker(self.state, self.y_gossip)
         if variant != B.DETAG_VARIANT_AUTO:
             B.detag_set_variant(self.state, variant)
+        if gradient_point != B.DETAG_GRADIENT_AT_NEW_MODEL:
+            B.detag_set_gradient_point(self.state, gradient_point)
 
     # ---- data movement (plumbing only)
     def upload(self, name: str, host) -> None:

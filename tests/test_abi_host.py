@@ -125,3 +125,34 @@ def test_state_accessors_without_device():
             B.detag_set_noise(st, -1.0, 0)
     finally:
         B.detag_destroy(st)
+
+
+def test_phase_length_matches_theorem_3_and_the_oracle():
+    import math
+
+    from oracle import detag_oracle as orc
+
+    lam_ring = (1.0 + 2.0 * math.cos(2.0 * math.pi / 256)) / 3.0
+    cases = [(16, 0.75, 0.0, 0.0, 1.0), (16, 0.75, 4.0, 1e6, 2.0), (2, 0.0, 0.0, 0.0, 1.0), (256, lam_ring, 0.0, 0.0, 1.0),
+             (64, 0.882843, 9.0, 5e4, 3.0)]
+    for case in cases:
+        assert B.detag_phase_length(*case) == orc.phase_length(*case), case
+    assert B.detag_phase_length(16, 0.75) == 3 and B.detag_phase_length(256, lam_ring) == 196
+    for bad in ((0, 0.5), (4, 1.0), (4, -0.1), (4, float("nan"))):
+        with pytest.raises(B.DetagError) as e:
+            B.detag_phase_length(*bad)
+        assert e.value.code == B.DETAG_ERR_ARG
+
+
+def test_gradient_point_accessors():
+    m = inputs.metropolis_weights(inputs.ring_graph(4))
+    st = B.detag_create(4, 16, m.row_ptr, m.col_idx, m.vals, 2, 0.1, 0.1)
+    try:
+        assert B.detag_get_gradient_point(st) == B.DETAG_GRADIENT_AT_NEW_MODEL
+        B.detag_set_gradient_point(st, B.DETAG_GRADIENT_AT_PHASE_START)
+        assert B.detag_get_gradient_point(st) == B.DETAG_GRADIENT_AT_PHASE_START
+        with pytest.raises(B.DetagError) as e:
+            B.detag_set_gradient_point(st, 7)
+        assert e.value.code == B.DETAG_ERR_ARG
+    finally:
+        B.detag_destroy(st)
