@@ -11,18 +11,22 @@
 // tracker and the model together, and because P is circulant the A fragment depends on s - 2t only:
 // ten doubles per lane, kept in registers, for every tile of the run.
 //
-// A CTA works on tiles (32 output rows x 64 coordinates).  Warp roles, mbarrier pipeline, padded TMA input
-// tiles (box = row pitch), dense output tile + TMA tile stores: as in the dense kernel for n <= 32.  The
-// window rows wrap around the ring, so the x, y windows are fetched as four 16-row boxes each at row
-// (R - 16 + 16 q) mod n; g, a, c are needed for the 32 output rows only.
+// A CTA owns whole slabs of 64 coordinates and walks the n/32 row blocks of a slab in order; one unit of work
+// ("tile") is 32 output rows x 64 coordinates.  Warp roles, mbarrier pipeline, padded TMA input tiles (box =
+// row pitch), dense output tile + TMA tile stores, tail inputs in registers and the stage handed back before
+// the tail: as in the dense kernel for n <= 32.  The window rows wrap around the ring, so the x, y windows are
+// fetched as four 16-row boxes each at row (R - 16 + 16 q) mod n; g, a, c are needed for the 32 output rows only.
+// The halo rows are read twice (once per neighbouring block); the second read comes from L2.
 //
-// The step updates x and y in place, and a tile's window contains rows that neighbouring row blocks
-// overwrite.  So the n/32 row blocks of one slab are processed by the CTAs of one thread-block cluster
-// (cluster rank = row block), and no CTA stores its results of a slab before every CTA of the cluster has
-// its window of that slab in shared memory: a signalling thread publishes "slab k landed" into a per-peer
-// counter in every peer's shared memory (st.release.cluster), and the storing thread polls its local copy of
-// all peers' counters before it issues the slab's TMA stores.  Halo rows of neighbouring row blocks are read
-// by CTAs of the same cluster at about the same time, so they come from L2.
+// The step updates x and y in place, and a tile's window contains rows that the neighbouring row blocks
+// overwrite.  Two rules keep every window on the old values:
+//   * the results of row block b are stored only after the window of block b+1 (which contains the last 16
+//     rows of block b) has landed in shared memory: a signalling thread publishes a "tiles landed" counter,
+//     and the storing thread (and the warps that write the d % 4 tail columns directly) wait for it;
+//   * the window of the last block ends with rows 0..15, which block 0 has overwritten long before: those
+//     rows are fetched into a side buffer together with block 0's window (before anything of the slab is
+//     stored) and the last block reads them from there.
+// Blocks further apart share no rows (n >= 64), and different slabs share no coordinates.
 //
 // Output rows are the natural blocks 8t + r (a permuted block would widen the band), so the four workers of
 // one Philox call sit in four lanes: each lane draws the calls of one block and a 4 x 4 transpose over those
@@ -54,12 +58,14 @@ constexpr int kGroupWarps = kS / 8;
 constexpr int kConsumerWarps = kGroupWarps * kWarpGroups;
 constexpr int kProducerWarp = kConsumerWarps, kStoreWarp = kConsumerWarps + 1, kSignalWarp = kConsumerWarps + 2;
 constexpr int kThreads = (kConsumerWarps + 3) * 32;
-constexpr int kMaxCluster = 8;     // portable cluster size: n <= 256
+constexpr int kSideFloats = 2 * kHalo * kPitchXY;  // rows 0..15 of x and y, kept for the slab's last row block
 constexpr int kOutFloats = 3 * kR * kS;
 constexpr int kBandSteps = 10;     // 4-row window steps that meet an 8-row output block: (2*16 + 8) / 4
 constexpr unsigned kSpinLimit = 1u << 20;
 constexpr unsigned kSuspendHintNs = 2000;
-constexpr size_t kSmemBytes = static_cast<size_t>(kStages) * kStageBytes + kWarpGroups * kOutFloats * 4 + 128;  // barriers + peer counters
+constexpr size_t kSmemBytes =
+    static_cast<size_t>(kStages) * kStageBytes + 2 * kSideFloats * 4 + kWarpGroups * kOutFloats * 4 + 128;  // + barriers, counters
+static_assert(kSmemBytes <= 232448, "shared memory plan");
 
 struct BandMaps {
   CUtensorMap x16, y16;        // loads, 16-row boxes of width kPitchXY
@@ -85,38 +91,6 @@ __device__ __forceinline__ bool bar_wait(uint64_t* bar, unsigned parity) {
         : "r"(addr), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     if (done) return true;
-  }
-  return false;
-}
-
-__device__ __forceinline__ unsigned cluster_rank() {
-  unsigned v;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(v));
-  return v;
-}
-
-__device__ __forceinline__ void cluster_sync_all() {  // every thread of every CTA of the cluster
-  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
-}
-
-// Writes `value` into the counter at the same shared-memory offset in CTA `peer` of the cluster.
-__device__ __forceinline__ void publish_to_peer(unsigned* local_counter, unsigned peer, unsigned value) {
-  uint32_t remote;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(s_addr(local_counter)), "r"(peer));
-  asm volatile("st.release.cluster.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"(value) : "memory");
-}
-
-// Bounded wait until all `count` counters (written by the peers) have reached `at_least`.
-__device__ __forceinline__ bool peers_wait(const unsigned* counters, int count, unsigned at_least) {
-  for (unsigned spin = 0; spin < kSpinLimit; ++spin) {
-    bool all = true;
-    for (int q = 0; q < count; ++q) {
-      unsigned v;
-      asm volatile("ld.acquire.cluster.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(s_addr(counters + q)) : "memory");
-      all = all && v >= at_least;
-    }
-    if (all) return true;
-    __nanosleep(200);
   }
   return false;
 }
@@ -185,20 +159,23 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
   // No static shared memory: the dynamic array starts at the CTA's shared window; its alignment is checked.
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* stage_mem = reinterpret_cast<float*>(smem_raw);
-  float* out_mem = stage_mem + kStages * kStageFloats;  // [group][x', y', g'][32][kS]
+  float* side_mem = stage_mem + kStages * kStageFloats;  // [slab parity][x, y][16][kPitchXY]
+  float* out_mem = side_mem + 2 * kSideFloats;           // [group][x', y', g'][32][kS]
   uint64_t* full = reinterpret_cast<uint64_t*>(out_mem + kWarpGroups * kOutFloats);
   uint64_t* empty = full + kStages;
   uint64_t* out_ready = empty + kStages;
   uint64_t* out_free = out_ready + kWarpGroups;
-  unsigned* landed = reinterpret_cast<unsigned*>(out_free + kWarpGroups);  // [peer]: slabs whose window peer has loaded
-  unsigned* seen = landed + kMaxCluster;  // [group]: 1 + index of the last slab whose data the group has seen
+  unsigned* landed = reinterpret_cast<unsigned*>(out_free + kWarpGroups);  // tiles whose window is in shared memory
+  unsigned* seen = landed + 1;  // [group]: 1 + index of the last tile whose data the group has seen
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = p.n;
-  const int row_blocks = n / kR;             // = cluster size
-  const int rb = static_cast<int>(cluster_rank());
-  const bool aligned_ok = (s_addr(smem_raw) & 127u) == 0;
+  const int row_blocks = n / kR;
+  if ((s_addr(smem_raw) & 127u) != 0) {
+    if (tid == 0) atomicExch(p.status, 2);
+    return;
+  }
   if (tid == 0) {
-    for (int q = 0; q < kMaxCluster; ++q) landed[q] = 0;
+    *landed = 0;
     for (int g = 0; g < kWarpGroups; ++g) seen[g] = 0;
     for (int s = 0; s < kStages; ++s) {
       bar_init(&full[s], 1);
@@ -209,48 +186,62 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
       bar_init(&out_free[g], 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    if (!aligned_ok) atomicExch(p.status, 2);
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  cluster_sync_all();  // counters and barriers of every CTA of the cluster are initialised
+  __syncthreads();
 
-  // the cluster takes slabs first, first + stride, ...; this CTA their row block rb
-  const long long first = blockIdx.x / row_blocks, stride = gridDim.x / row_blocks;
-  const long long num_tiles = aligned_ok ? p.num_slabs : 0;  // "tile" below = slab of this cluster
+  // this CTA takes slabs blockIdx.x, blockIdx.x + gridDim.x, ...; tile k is row block k % row_blocks of its
+  // (k / row_blocks)-th slab
+  const long long my_slabs = blockIdx.x < p.num_slabs ? (p.num_slabs - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+  const long long num_tiles = my_slabs * row_blocks;
 
   if (warp == kSignalWarp) {
-    // tells every CTA of the cluster (itself included) that this CTA's window of slab k is in shared memory
+    // publishes how many tiles (in order) have their window in shared memory
     if (lane == 0) {
-      long long k = 0;
-      for (long long tile = first; tile < num_tiles; tile += stride, ++k) {
+      for (long long k = 0; k < num_tiles; ++k) {
         const int s = static_cast<int>(k % kStages);
         if (!bar_wait(&full[s], (k / kStages) & 1)) {
           atomicExch(p.status, 1);
           break;
         }
-        for (int peer = 0; peer < row_blocks; ++peer) publish_to_peer(&landed[rb], peer, static_cast<unsigned>(k + 1));
+        count_publish(landed, static_cast<unsigned>(k + 1));
         bar_arrive(&empty[s]);  // keeps the stage's phase from running ahead of this thread
       }
     }
-  } else if (warp == kProducerWarp) {
+    return;
+  }
+  if (warp == kProducerWarp) {
     if (lane == 0) {
-      int issued = 0;
+      long long issued = 0;
       bool ok = true;
-      for (long long tile = first; tile < num_tiles; tile += stride, ++issued) {
-        const int s = issued % kStages;
+      for (; issued < num_tiles; ++issued) {
+        const int s = static_cast<int>(issued % kStages);
         if (issued >= kStages) ok = bar_wait(&empty[s], ((issued / kStages) - 1) & 1);
         if (!ok) break;
-        const long long slab = tile;
+        const long long slab_no = issued / row_blocks;
+        const int rb = static_cast<int>(issued % row_blocks);
+        const long long slab = blockIdx.x + slab_no * gridDim.x;
         float* st = stage_mem + static_cast<size_t>(s) * kStageFloats;
         const int col = static_cast<int>(slab * kS);
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_addr(&full[s])),
-                     "r"(static_cast<unsigned>(kStageBytes))
+        const bool last = rb == row_blocks - 1;
+        // the last block's final window piece (rows 0..15) is not loaded: it comes from the side buffer
+        const unsigned bytes = static_cast<unsigned>(kStageBytes) - (last ? 2u * 16 * kPitchXY * 4 : 0u) +
+                               (rb == 0 ? static_cast<unsigned>(kSideFloats) * 4 : 0u);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_addr(&full[s])), "r"(bytes)
                      : "memory");
 #pragma unroll
         for (int q = 0; q < kW / 16; ++q) {  // the window wraps around the ring in 16-row pieces
+          if (last && q == kW / 16 - 1) continue;
           const int row = ((rb * kR - kHalo + 16 * q) % n + n) % n;
           tile_load(st + q * 16 * kPitchXY, &maps.x16, col, row, &full[s]);
           tile_load(st + kW * kPitchXY + q * 16 * kPitchXY, &maps.y16, col, row, &full[s]);
+        }
+        if (rb == 0) {
+          // Rows 0..15 before anything of this slab is stored.  The buffer of this parity was last read by the
+          // last block of the slab before the previous one, whose stage has been recycled since.
+          float* sd = side_mem + static_cast<size_t>(slab_no & 1) * kSideFloats;
+          tile_load(sd, &maps.x16, col, 0, &full[s]);
+          tile_load(sd + kHalo * kPitchXY, &maps.y16, col, 0, &full[s]);
         }
         float* se = st + 2 * kW * kPitchXY;
 #pragma unroll
@@ -263,29 +254,31 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
       }
       if (!ok) {
         atomicExch(p.status, 1);
-        for (int back = 1; back <= kStages && back <= issued; ++back) {  // drain copies still in flight (bounded)
-          const int k = issued - back;
+        for (long long back = 1; back <= kStages && back <= issued; ++back) {  // drain copies still in flight (bounded)
+          const long long k = issued - back;
           bar_wait(&full[k % kStages], (k / kStages) & 1);
         }
       }
     }
-  } else if (warp == kStoreWarp) {
+    return;
+  }
+  if (warp == kStoreWarp) {
     if (lane == 0) {
-      long long k = 0;
-      for (long long tile = first; tile < num_tiles; tile += stride, ++k) {
+      for (long long k = 0; k < num_tiles; ++k) {
         const int g = static_cast<int>(k % kWarpGroups);
         if (!bar_wait(&out_ready[g], (k / kWarpGroups) & 1)) {
           atomicExch(p.status, 1);
           break;
         }
-        const long long slab = tile;
-        // in-place update: every CTA of the cluster must hold its window of this slab before anyone overwrites it
-        if (!peers_wait(landed, row_blocks, static_cast<unsigned>(k + 1))) {
+        const long long slab_no = k / row_blocks;
+        const int rb = static_cast<int>(k % row_blocks);
+        // in-place update: the next block's window (it contains this block's last rows) must have landed
+        if (rb + 1 < row_blocks && !count_wait(landed, static_cast<unsigned>(k + 2))) {
           atomicExch(p.status, 1);
           break;
         }
         const float* ob = out_mem + g * kOutFloats;
-        const int col = static_cast<int>(slab * kS);
+        const int col = static_cast<int>((blockIdx.x + slab_no * gridDim.x) * kS);
         if (col < (p.d & ~3LL)) {
           tile_store(&maps.xs, col, rb * kR, ob);
           tile_store(&maps.ys, col, rb * kR, ob + kR * kS);
@@ -297,7 +290,9 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
       }
       asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
-  } else {
+    return;
+  }
+
   // ------------------------------------------------------------------ consumer warps
   const int r = lane >> 2, kq = lane & 3;
   const int group = warp / kGroupWarps, mtile = warp % kGroupWarps;
@@ -316,10 +311,14 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
   }
   const int pos = r & 3, half = r >> 2;  // this lane's worker is number `pos` of its Philox quad
 
-  long long use = 0;
-  for (long long k = group, tile = first + group * stride; tile < num_tiles;
-       tile += kWarpGroups * stride, k += kWarpGroups, ++use) {
-    const int s = static_cast<int>(k % kStages);
+  // 32-bit bookkeeping: the launcher admits this kernel only for d < 2^31, so tile and slab counts fit easily
+  const int tiles = static_cast<int>(num_tiles);
+  int use = 0;
+  for (int k = group; k < tiles; k += kWarpGroups, ++use) {
+    const int s = k % kStages;
+    const int slab_no = k / row_blocks;
+    const int rb = k - slab_no * row_blocks;
+    const long long slab = blockIdx.x + static_cast<long long>(slab_no) * gridDim.x;
     bool ok = true;
     if (lane == 0) {
       // with an odd stage count the stage last served the other group: a parity wait must not start before
@@ -328,28 +327,31 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
         ok = count_wait(&seen[(k - kStages) % kWarpGroups], static_cast<unsigned>(k - kStages + 1));
       if (ok) ok = bar_wait(&full[s], (k / kStages) & 1);
       if (ok && mtile == 0) count_publish(&seen[group], static_cast<unsigned>(k + 1));
-      if (ok && use > 0) ok = bar_wait(&out_free[group], (use - 1) & 1);
     }
-    const long long slab = tile;
-    // the d % 4 tail columns are stored directly (not by the storing thread): same in-place rule for them
-    if (lane == 0 && ok && slab * kS + kS > d_tma && p.d != d_tma)
-      ok = peers_wait(landed, row_blocks, static_cast<unsigned>(k + 1));
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     if (!ok) {
       if (lane == 0) atomicExch(p.status, 1);
-      break;
+      return;
     }
     const float* sx = stage_mem + static_cast<size_t>(s) * kStageFloats;
     const float* sy = sx + kW * kPitchXY;
     const float* sg = sy + kW * kPitchXY;
     const float* sa = sg + kR * kPitchE;
     const float* sc = sa + kR * kPitchE;
+    // window rows 48..63 of the slab's last block are rows 0..15 of the ring: kept in the side buffer
+    const bool wrap_side = rb == row_blocks - 1;
+    // offsets (in floats, relative to sx / sy) that redirect window rows 48..63 to the side buffer
+    const int side_dx = static_cast<int>(side_mem + (slab_no & 1) * kSideFloats - sx) - (kW - kHalo) * kPitchXY;
+    const int side_dy = side_dx + kHalo * kPitchXY - kW * kPitchXY;
     const long long j0 = slab * kS;
+    const long long j = j0 + cl + 2 * kq;
+    const bool active = j0 + cl < p.d;  // a tile wholly beyond column d computes nothing but keeps the protocol
 
-    if (j0 + cl < p.d) {
-      // cx accumulates P (x - alpha y) = x' and cy starts at -g, ending as y~ - g: the tail then needs a single
-      // float64 addition (scalar float64 work queues behind other warps' MMAs on the shared FP64 pipe)
-      double cy[4][2], cx[4][2];
+    // cx accumulates P (x - alpha y) = x' and cy starts at -g, ending as y~ - g: the tail then needs a single
+    // float64 addition (scalar float64 work queues behind other warps' MMAs on the shared FP64 pipe)
+    double cy[4][2], cx[4][2];
+    float2 av4[4], cv4[4];
+    if (active) {
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const float2 gv = *reinterpret_cast<const float2*>(sg + (8 * t + r) * kPitchE + cl + 2 * kq);
@@ -360,8 +362,9 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
 #pragma unroll
       for (int ws = 0; ws < kW / 4; ++ws) {  // window steps of four rows
         const int src = (4 * ws + kq) * kPitchXY + cl + r;
-        const double by = static_cast<double>(sy[src]);
-        const double bx = fma(-alpha, by, static_cast<double>(sx[src]));
+        const bool side = ws >= (kW - kHalo) / 4 && wrap_side;
+        const double by = static_cast<double>(sy[src + (side ? side_dy : 0)]);
+        const double bx = fma(-alpha, by, static_cast<double>(sx[src + (side ? side_dx : 0)]));
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
           const int u = ws - 2 * t;  // compile-time after unrolling: only the band's blocks are issued
@@ -371,9 +374,31 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
           }
         }
       }
+      // the tail's inputs move to registers so that the stage can be refilled while the tail runs
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int eoff = (8 * t + r) * kPitchE + cl + 2 * kq;
+        av4[t] = *reinterpret_cast<const float2*>(sa + eoff);
+        cv4[t] = *reinterpret_cast<const float2*>(sc + eoff);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) {
+      bar_arrive(&empty[s]);  // stage no longer read by this warp
+      if (use > 0) ok = bar_wait(&out_free[group], (use - 1) & 1);  // previous tile of this group stored
+      // the d % 4 tail columns are stored directly (not by the storing thread): same in-place rule for them
+      if (ok && j0 + kS > d_tma && p.d != d_tma && rb + 1 < row_blocks)
+        ok = count_wait(landed, static_cast<unsigned>(k + 2));
+    }
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    if (!ok) {
+      if (lane == 0) atomicExch(p.status, 1);
+      return;
+    }
+
+    if (active) {
       // noise: this lane draws the two calls (coordinates j, j+1) of block t = pos for its half, then the
       // 4 x 4 transposes over the lanes of the quad give it the normals of its own worker for t = 0..3
-      const long long j = j0 + cl + 2 * kq;
       float xi[2][4];
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
@@ -389,16 +414,17 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const int orow = 8 * t + r;  // output row within the tile
-        const int eoff = orow * kPitchE + cl + 2 * kq;
-        const float2 av = *reinterpret_cast<const float2*>(sa + eoff);
-        const float2 cv = *reinterpret_cast<const float2*>(sc + eoff);
+        const float2 av = av4[t], cv = cv4[t];
         float2 xo, yo, go;
         xo.x = static_cast<float>(cx[t][0]);                              // x' (Algorithm 2's model update)
         xo.y = static_cast<float>(cx[t][1]);
-        float2 x_at = xo;  // gradient point: the new model, or (Algorithm 2 as printed) the model before this step,
-        if (p.grad_at_start) {  // which sits in the window: output row orow is window row orow + kHalo
-          const float* xw = sx + (orow + kHalo) * kPitchXY + cl + 2 * kq;
-          x_at = make_float2(xw[0], xw[1]);
+        const long long off = static_cast<long long>(rb * kR + orow) * p.ld + j;
+        // Gradient point: the new model, or (Algorithm 2 as printed) the model before this step.  The old x and g
+        // of this tile are still in global memory: its stores are issued after all of its warps are done.
+        float2 x_at = xo;
+        if (p.grad_at_start) {
+          x_at.x = j < p.d ? p.x[off] : 0.f;
+          x_at.y = j + 1 < p.d ? p.x[off + 1] : 0.f;
         }
         go.x = fmaf(av.x, x_at.x - cv.x, sigma * xi[0][t]);               // stochastic gradient
         go.y = fmaf(av.y, x_at.y - cv.y, sigma * xi[1][t]);
@@ -408,7 +434,10 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
         *reinterpret_cast<float2*>(ob + ooff) = xo;
         *reinterpret_cast<float2*>(ob + kR * kS + ooff) = yo;
         *reinterpret_cast<float2*>(ob + 2 * kR * kS + ooff) = go;
-        const long long off = static_cast<long long>(rb * kR + orow) * p.ld + j;
+        if (p.y_obs != nullptr) {  // optional observer: the gossiped tracker y~ = (y~ - g) + g, stored directly
+          if (j < p.d) p.y_obs[off] = static_cast<float>(cy[t][0] + static_cast<double>(p.g[off]));
+          if (j + 1 < p.d) p.y_obs[off + 1] = static_cast<float>(cy[t][1] + static_cast<double>(p.g[off + 1]));
+        }
         if (j >= d_tma) {  // the last d % 4 coordinates: TMA clips stores at 16-byte granularity
           if (j < p.d) {
             p.x[off] = xo.x;
@@ -421,33 +450,18 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
             p.g[off + 1] = go.y;
           }
         }
-        if (p.y_obs != nullptr) {  // optional observer: the gossiped tracker, stored directly
-          const float2 gv = *reinterpret_cast<const float2*>(sg + eoff);
-          if (j + 1 < p.d) {
-            *reinterpret_cast<float2*>(p.y_obs + off) =
-                make_float2(static_cast<float>(cy[t][0] + static_cast<double>(gv.x)),
-                            static_cast<float>(cy[t][1] + static_cast<double>(gv.y)));
-          } else if (j < p.d) {
-            p.y_obs[off] = static_cast<float>(cy[t][0] + static_cast<double>(gv.x));
-          }
-        }
       }
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // outputs visible to the TMA store
     __syncwarp();
-    if (lane == 0) {
-      bar_arrive(&out_ready[group]);
-      bar_arrive(&empty[s]);
-    }
+    if (lane == 0) bar_arrive(&out_ready[group]);
   }
-  }
-  cluster_sync_all();  // no CTA leaves while a peer may still write its counters
 }
 
 }  // namespace
 
 bool band_variant_available(int n, int half_band) {
-  return n % kR == 0 && n >= kW && n / kR <= kMaxCluster && half_band <= kHalo && encode_tiled_fn() != nullptr;
+  return n % kR == 0 && n >= kW && n <= kMaxWorkers && half_band <= kHalo && encode_tiled_fn() != nullptr;
 }
 
 int launch_step_band(StepParams p, const double* band /* 2*16+1 entries, p(delta) at index delta+16 */, int sm_count,
@@ -469,31 +483,10 @@ int launch_step_band(StepParams p, const double* band /* 2*16+1 entries, p(delta
   cudaError_t e = cudaFuncSetAttribute(step_band_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(kSmemBytes));
   if (e != cudaSuccess) return static_cast<int>(e);
-  e = cudaFuncSetAttribute(step_band_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 0);
-  if (e != cudaSuccess) return static_cast<int>(e);
-  const int row_blocks = p.n / kR;  // = cluster size: the CTAs of a cluster take the row blocks of one slab
-  cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = static_cast<unsigned>(row_blocks);
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = kSmemBytes;
-  cfg.stream = stream;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cfg.gridDim = dim3(static_cast<unsigned>(row_blocks));
-  int max_clusters = 0;
-  e = cudaOccupancyMaxActiveClusters(&max_clusters, step_band_kernel, &cfg);
-  if (e != cudaSuccess) return static_cast<int>(e);
-  if (max_clusters < 1) return static_cast<int>(cudaErrorLaunchOutOfResources);
-  (void)sm_count;
-  const long long clusters = p.num_slabs < max_clusters ? p.num_slabs : max_clusters;
-  if (clusters <= 0) return 0;
-  cfg.gridDim = dim3(static_cast<unsigned>(clusters * row_blocks));
-  e = cudaLaunchKernelEx(&cfg, step_band_kernel, p, maps, coef);
-  return static_cast<int>(e != cudaSuccess ? e : cudaGetLastError());
+  const long long grid = p.num_slabs < sm_count ? p.num_slabs : sm_count;
+  if (grid <= 0) return 0;
+  step_band_kernel<<<static_cast<unsigned>(grid), kThreads, kSmemBytes, stream>>>(p, maps, coef);
+  return static_cast<int>(cudaGetLastError());
 }
 
 }  // namespace detag
