@@ -176,7 +176,7 @@ int launch_step(detag_state* s, StepParams& p, cudaStream_t stream) {
   switch (resolve_variant(s)) {
     case DETAG_VARIANT_DENSE:
       e = p.n <= 32 ? detag::launch_step_mma(p, s->sm_count, stream)
-                    : detag::launch_step_dense(p, s->sm_count, stream);
+                    : detag::launch_step_band(p, nullptr, s->sm_count, stream);
       break;
     case DETAG_VARIANT_RING:
       e = detag::launch_step_band(p, s->band, s->sm_count, stream);

@@ -60,10 +60,10 @@ int launch_init_gradient(const StepParams& p, int sm_count, cudaStream_t stream)
 int plan_step_csr(StepParams& p, int smem_optin_bytes);  // chooses S; DETAG_ERR_UNSUPPORTED if nothing fits
 int launch_step_csr(const StepParams& p, int sm_count, cudaStream_t stream);
 bool dense_variant_available(int n);  // n <= kMaxDenseWorkers and the driver offers tensor-map encoding
-int launch_step_dense(const StepParams& p, int sm_count, cudaStream_t stream);  // register-tiled, 32 < n <= 64
 int launch_step_mma(StepParams p, int sm_count, cudaStream_t stream);           // FP64 tensor path, n <= 32
 bool band_variant_available(int n, int half_band);  // circulant band kernel: n % 32 == 0, n >= 64, half-band <= 16
-int launch_step_band(StepParams p, const double* band, int sm_count, cudaStream_t stream);
+bool dense_window_available(int n);                // the band kernel's dense mode: 32 < n <= 64
+int launch_step_band(StepParams p, const double* band /* null: dense mode */, int sm_count, cudaStream_t stream);
 int launch_consensus_error(const StepParams& p, double* partials, double* result, int sm_count, cudaStream_t stream);
 
 }  // namespace detag

@@ -28,6 +28,12 @@
 //     stored) and the last block reads them from there.
 // Blocks further apart share no rows (n >= 64), and different slabs share no coordinates.
 //
+// Dense mode (template flag): for 32 < n <= 64 the same machinery applies the full polynomial P_K(M) of any gossip
+// matrix.  The window is then simply rows 0..63 (all workers; rows >= n are zero-filled by the loads) for both
+// row blocks, every one of the 16 x 4 blocks of the 32 x 64 slice of P is issued (128 MMAs per tile), and the A
+// fragments come from shared memory (32 KB for the two slices) instead of ten registers.  No rows wrap, so the
+// side buffer is idle; the first in-place rule is all that is needed.
+//
 // Output rows are the natural blocks 8t + r (a permuted block would widen the band), so the four workers of
 // one Philox call sit in four lanes: each lane draws the calls of one block and a 4 x 4 transpose over those
 // lanes (two shuffle stages) hands every lane its own workers' normals.
@@ -65,7 +71,8 @@ constexpr unsigned kSpinLimit = 1u << 20;
 constexpr unsigned kSuspendHintNs = 2000;
 constexpr size_t kSmemBytes =
     static_cast<size_t>(kStages) * kStageBytes + 2 * kSideFloats * 4 + kWarpGroups * kOutFloats * 4 + 128;  // + barriers, counters
-static_assert(kSmemBytes <= 232448, "shared memory plan");
+constexpr int kDenseFragBytes = 2 * (kW / 4) * 4 * 32 * 8;  // dense mode: [row block][window step][t][lane] doubles
+static_assert(kSmemBytes + kDenseFragBytes <= 232448, "shared memory plan");
 
 struct BandMaps {
   CUtensorMap x16, y16;        // loads, 16-row boxes of width kPitchXY
@@ -154,6 +161,7 @@ __device__ __forceinline__ void transpose4(float (&v)[4], int q) {
   if (b1) { v[0] = r0; v[1] = r1; } else { v[2] = r0; v[3] = r1; }
 }
 
+template <bool kDense>
 __global__ void __launch_bounds__(kThreads, 1)
 step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, const __grid_constant__ BandCoef coef) {
   // No static shared memory: the dynamic array starts at the CTA's shared window; its alignment is checked.
@@ -167,12 +175,21 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
   uint64_t* out_free = out_ready + kWarpGroups;
   unsigned* landed = reinterpret_cast<unsigned*>(out_free + kWarpGroups);  // tiles whose window is in shared memory
   unsigned* seen = landed + 1;  // [group]: 1 + index of the last tile whose data the group has seen
+  double* frag = reinterpret_cast<double*>(smem_raw + kSmemBytes);  // dense mode only (the launch adds the bytes)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = p.n;
-  const int row_blocks = n / kR;
+  const int row_blocks = kDense ? 2 : n / kR;
   if ((s_addr(smem_raw) & 127u) != 0) {
     if (tid == 0) atomicExch(p.status, 2);
     return;
+  }
+  if (kDense) {
+    // slice rb of P in fragment order: block (ws, t), lane (r, kq) holds P[32 rb + 8t + r][4 ws + kq]
+    for (int e = tid; e < 2 * (kW / 4) * 4 * 32; e += kThreads) {
+      const int l = e & 31, t = (e >> 5) & 3, ws = (e >> 7) % (kW / 4), b = e / (32 * 4 * (kW / 4));
+      const int i = kR * b + 8 * t + (l >> 2), j = 4 * ws + (l & 3);
+      frag[e] = (i < n && j < n) ? p.poly[static_cast<size_t>(i) * n + j] : 0.0;
+    }
   }
   if (tid == 0) {
     *landed = 0;
@@ -223,20 +240,20 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
         const long long slab = blockIdx.x + slab_no * gridDim.x;
         float* st = stage_mem + static_cast<size_t>(s) * kStageFloats;
         const int col = static_cast<int>(slab * kS);
-        const bool last = rb == row_blocks - 1;
+        const bool last = !kDense && rb == row_blocks - 1;
         // the last block's final window piece (rows 0..15) is not loaded: it comes from the side buffer
         const unsigned bytes = static_cast<unsigned>(kStageBytes) - (last ? 2u * 16 * kPitchXY * 4 : 0u) +
-                               (rb == 0 ? static_cast<unsigned>(kSideFloats) * 4 : 0u);
+                               (!kDense && rb == 0 ? static_cast<unsigned>(kSideFloats) * 4 : 0u);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_addr(&full[s])), "r"(bytes)
                      : "memory");
 #pragma unroll
         for (int q = 0; q < kW / 16; ++q) {  // the window wraps around the ring in 16-row pieces
           if (last && q == kW / 16 - 1) continue;
-          const int row = ((rb * kR - kHalo + 16 * q) % n + n) % n;
+          const int row = kDense ? 16 * q : ((rb * kR - kHalo + 16 * q) % n + n) % n;
           tile_load(st + q * 16 * kPitchXY, &maps.x16, col, row, &full[s]);
           tile_load(st + kW * kPitchXY + q * 16 * kPitchXY, &maps.y16, col, row, &full[s]);
         }
-        if (rb == 0) {
+        if (!kDense && rb == 0) {
           // Rows 0..15 before anything of this slab is stored.  The buffer of this parity was last read by the
           // last block of the slab before the previous one, whose stage has been recycled since.
           float* sd = side_mem + static_cast<size_t>(slab_no & 1) * kSideFloats;
@@ -303,11 +320,13 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
   const int cl = mtile * 8;
   const long long d_tma = p.d & ~3LL;
   // A fragment of window step u = s - 2t: element [r][kq] = p(4u + kq - r - 16); the same for every block and tile
-  double afrag[kBandSteps];
+  double afrag[kDense ? 1 : kBandSteps];
+  if (!kDense) {
 #pragma unroll
-  for (int u = 0; u < kBandSteps; ++u) {
-    const int delta = 4 * u + kq - r - kHalo;
-    afrag[u] = (delta >= -kHalo && delta <= kHalo) ? coef.p[delta + kHalo] : 0.0;
+    for (int u = 0; u < kBandSteps; ++u) {
+      const int delta = 4 * u + kq - r - kHalo;
+      afrag[u] = (delta >= -kHalo && delta <= kHalo) ? coef.p[delta + kHalo] : 0.0;
+    }
   }
   const int pos = r & 3, half = r >> 2;  // this lane's worker is number `pos` of its Philox quad
 
@@ -339,7 +358,7 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
     const float* sa = sg + kR * kPitchE;
     const float* sc = sa + kR * kPitchE;
     // window rows 48..63 of the slab's last block are rows 0..15 of the ring: kept in the side buffer
-    const bool wrap_side = rb == row_blocks - 1;
+    const bool wrap_side = !kDense && rb == row_blocks - 1;
     // offsets (in floats, relative to sx / sy) that redirect window rows 48..63 to the side buffer
     const int side_dx = static_cast<int>(side_mem + (slab_no & 1) * kSideFloats - sx) - (kW - kHalo) * kPitchXY;
     const int side_dy = side_dx + kHalo * kPitchXY - kW * kPitchXY;
@@ -367,10 +386,16 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
         const double bx = fma(-alpha, by, static_cast<double>(sx[src + (side ? side_dx : 0)]));
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-          const int u = ws - 2 * t;  // compile-time after unrolling: only the band's blocks are issued
-          if (u >= 0 && u < kBandSteps) {
-            dmma(cy[t], afrag[u], by);
-            dmma(cx[t], afrag[u], bx);
+          if (kDense) {
+            const double a = frag[((rb * (kW / 4) + ws) * 4 + t) * 32 + lane];
+            dmma(cy[t], a, by);
+            dmma(cx[t], a, bx);
+          } else {
+            const int u = ws - 2 * t;  // compile-time after unrolling: only the band's blocks are issued
+            if (u >= 0 && u < kBandSteps) {
+              dmma(cy[t], afrag[u], by);
+              dmma(cx[t], afrag[u], bx);
+            }
           }
         }
       }
@@ -464,11 +489,17 @@ bool band_variant_available(int n, int half_band) {
   return n % kR == 0 && n >= kW && n <= kMaxWorkers && half_band <= kHalo && encode_tiled_fn() != nullptr;
 }
 
-int launch_step_band(StepParams p, const double* band /* 2*16+1 entries, p(delta) at index delta+16 */, int sm_count,
-                     cudaStream_t stream) {
+bool dense_window_available(int n) { return n > kR && n <= kW && encode_tiled_fn() != nullptr; }
+
+bool dense_variant_available(int n) { return n >= 1 && n <= kMaxDenseWorkers && encode_tiled_fn() != nullptr; }
+
+// band == nullptr: dense mode (32 < n <= 64, p.poly holds P_K(M)); otherwise the circulant band of 2*16+1 entries,
+// p(delta) at index delta + 16.
+int launch_step_band(StepParams p, const double* band, int sm_count, cudaStream_t stream) {
   BandMaps maps;
   BandCoef coef;
-  for (int k = 0; k < 2 * kHalo + 1; ++k) coef.p[k] = band[k];
+  const bool dense = band == nullptr;
+  for (int k = 0; k < 2 * kHalo + 1; ++k) coef.p[k] = dense ? 0.0 : band[k];
   const long long d_tma = p.d & ~3LL;
   if (!make_map(&maps.x16, p.x, p.n, p.d, p.ld, 16, kPitchXY) || !make_map(&maps.y16, p.y, p.n, p.d, p.ld, 16, kPitchXY) ||
       !make_map(&maps.g16, p.g, p.n, p.d, p.ld, 16, kPitchE) || !make_map(&maps.a16, p.a, p.n, p.d, p.ld, 16, kPitchE) ||
@@ -480,12 +511,13 @@ int launch_step_band(StepParams p, const double* band /* 2*16+1 entries, p(delta
   if (d_tma == 0) maps.xs = maps.ys = maps.gs = maps.x16;  // never used
   p.S = kS;
   p.num_slabs = (p.d + kS - 1) / kS;
-  cudaError_t e = cudaFuncSetAttribute(step_band_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(kSmemBytes));
+  auto kernel = dense ? step_band_kernel<true> : step_band_kernel<false>;
+  const size_t smem = kSmemBytes + (dense ? kDenseFragBytes : 0);
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return static_cast<int>(e);
   const long long grid = p.num_slabs < sm_count ? p.num_slabs : sm_count;
   if (grid <= 0) return 0;
-  step_band_kernel<<<static_cast<unsigned>(grid), kThreads, kSmemBytes, stream>>>(p, maps, coef);
+  kernel<<<static_cast<unsigned>(grid), kThreads, smem, stream>>>(p, maps, coef);
   return static_cast<int>(cudaGetLastError());
 }
 
