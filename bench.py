@@ -34,18 +34,36 @@ BYTES_PER_WC = 32  # read x, y, g, a, c + write x, y, g, float32 each: the fused
 # small case of the same kernel; traffic grows in proportion to n*d).  Keyed by the sha256 prefix of the kernel
 # source the capture was taken on: a changed kernel reports null until it is captured again.
 MEASURED_TRAFFIC = {
-    "step_mma.cu": ("1f9c10577c38a0a4", 31.29),   # cfg5 shape, d = 2,000,000: 1.2835 GB read + 0.7189 GB written / 64 M wc
-    "step_band.cu": ("2fac1dfc9e253737", 31.10),  # cfg4 shape, d = 200,000: 1.0244 GB read + 0.5681 GB written / 51.2 M wc
+    # cfg5 shape, d = 2,000,000: 1.2854 GB read + 0.7178 GB written / 64 M wc
+    ("step_mma.cu", "dense"): ("996d4601c5b9033f", 31.30),
+    # cfg4 shape, d = 200,000: 1.0270 GB read + 0.5706 GB written / 51.2 M wc (the re-read halo rows come from L2)
+    ("step_band.cu", "ring"): ("ef85fb13d585b2ae", 31.20),
+    # cfg3 shape, d = 500,000: 0.6447 GB read + 0.3369 GB written / 32 M wc
+    ("step_band.cu", "dense"): ("ef85fb13d585b2ae", 30.68),
 }
+
+# Float64 multiply-adds per worker-coordinate on the FP64 tensor pipe (both contractions, padded shapes) and that
+# pipe's peak: 64 multiply-adds per clock and SM (measured: 61 with m8n8k4 MMAs from 16 warps) x 148 SMs x max clock.
+FP64_FMA_PER_WC = {("step_mma.cu", "dense"): 64, ("step_band.cu", "ring"): 80, ("step_band.cu", "dense"): 128}
+FP64_FMA_PER_CLK_SM = 64
+SM_COUNT = 148
+
+
+def kernel_key(variant: str, n: int):
+    if variant == "dense":
+        return ("step_mma.cu", "dense") if n <= 32 else ("step_band.cu", "dense")
+    if variant == "ring":
+        return ("step_band.cu", "ring")
+    return None
 
 
 def measured_traffic_bytes(variant: str, n: int, wc: int):
     import hashlib
-    name = {"dense": "step_mma.cu" if n <= 32 else None, "ring": "step_band.cu"}.get(variant)
-    if name is None:
+    key = kernel_key(variant, n)
+    if key is None:
         return None
-    digest, per_wc = MEASURED_TRAFFIC[name]
-    path = os.path.join(ROOT, "paper_2006_08085_b200", "csrc", name)
+    digest, per_wc = MEASURED_TRAFFIC[key]
+    path = os.path.join(ROOT, "paper_2006_08085_b200", "csrc", key[0])
     try:
         with open(path, "rb") as fh:
             if hashlib.sha256(fh.read()).hexdigest()[:16] != digest:
@@ -261,6 +279,13 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         kernel_ms = float(per_step.mean())
         achieved = BYTES_PER_WC * cfg.wc / (kernel_ms * 1e-3) / 1e9
         traffic = measured_traffic_bytes(variant, cfg.n, cfg.wc)
+        key = kernel_key(variant, cfg.n)
+        fp64 = None
+        if key is not None:  # second roofline: the FP64 tensor pipe that carries both contractions
+            fma = FP64_FMA_PER_WC[key] * cfg.wc / (kernel_ms * 1e-3)
+            fp64_peak = FP64_FMA_PER_CLK_SM * SM_COUNT * (clocks.get("sm_max_mhz") or 1965) * 1e6
+            fp64 = {"fma_per_wc": FP64_FMA_PER_WC[key], "achieved_tfma_s": fma / 1e12, "peak_tfma_s": fp64_peak / 1e12,
+                    "frac": fma / fp64_peak, "peak_source": "64 FMA/clk/SM x 148 SMs x max SM clock"}
         line = {
             "metric": METRIC, "value": world * cfg.wc * args.steps / (total_ms_max * 1e-3), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
@@ -274,7 +299,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "peak_source": peak_src, "bytes_per_wc": BYTES_PER_WC,
                          "kernel_ms": kernel_ms, "kernel_ms_min": float(per_step.min()),
-                         "frac_of_8TBps_nominal": achieved / 8000.0},
+                         "frac_of_8TBps_nominal": achieved / 8000.0, "fp64_tensor_pipe": fp64},
             "clocks": clocks,
             "gpu_launches": args.steps,
             "consensus_error_after_run": consensus,
