@@ -161,6 +161,16 @@ int detag_init(detag_state* s, void* stream);
 int detag_step(detag_state* s, void* stream);
 
 /*
+ * `count` consecutive DeTAG iterations: the same result, bit for bit, as `count` calls of detag_step.
+ * The iteration never mixes coordinates (Algorithm 3 mixes workers only, the synthetic objective is
+ * diagonal), so where the kernel variant allows it (dense polynomial, n <= 32, no observer buffer) all
+ * `count` iterations of a coordinate slab run on chip in one launch and the state crosses HBM once per
+ * call instead of once per iteration; otherwise the call enqueues `count` single steps.
+ * Asynchronous; the step counter advances by `count`.  Errors: ARG (count < 1), UNBOUND, CUDA.
+ */
+int detag_step_many(detag_state* s, int count, void* stream);
+
+/*
  * Consensus error of the model, ||X - Xbar 1^T||_F^2 = sum_j sum_i (x_ij - mean_i x_ij)^2
  * (the quantity bounded in the proof of Theorem 3), accumulated in float64 in a fixed order.
  * Enqueues on `stream`, waits for it, writes *host_out.  Errors: ARG, UNBOUND, CUDA.

@@ -61,6 +61,7 @@ SIGNATURES = {
                                           ctypes.c_double, ctypes.POINTER(ctypes.c_int)]),
     "detag_init": (ctypes.c_int, [_P, _P]),
     "detag_step": (ctypes.c_int, [_P, _P]),
+    "detag_step_many": (ctypes.c_int, [_P, ctypes.c_int, _P]),
     "detag_step_host": (ctypes.c_int, [_P, ctypes.c_int64, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P]),
     "detag_host_staging_bytes": (ctypes.c_int, [_P, ctypes.c_int64, ctypes.POINTER(ctypes.c_size_t)]),
     "detag_consensus_error": (ctypes.c_int, [_P, _P, _F64P]),
@@ -200,6 +201,11 @@ def detag_init(state, stream=None) -> None:
 
 def detag_step(state, stream=None) -> None:
     _check(lib().detag_step(state, _stream_handle(stream)), "detag_step", state)
+
+
+def detag_step_many(state, count: int, stream=None) -> None:
+    """`count` iterations; where the variant allows it they run on chip in one launch (same bits as detag_step)."""
+    _check(lib().detag_step_many(state, int(count), _stream_handle(stream)), "detag_step_many", state)
 
 
 def detag_step_host(state, ld_host: int, x, y, g, a, c, staging, staging_bytes: int, stream=None) -> None:

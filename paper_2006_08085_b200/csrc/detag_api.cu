@@ -388,6 +388,27 @@ int detag_step(detag_state* s, void* stream) {
   return DETAG_OK;
 }
 
+int detag_step_many(detag_state* s, int count, void* stream) {
+  if (!s) return DETAG_ERR_ARG;
+  if (count < 1) return fail(s, DETAG_ERR_ARG, "detag_step_many: count must be at least 1");
+  if (!s->bound) return fail(s, DETAG_ERR_UNBOUND, "detag_step_many before detag_bind");
+  // the fused kernel exists for the dense polynomial with n <= 32; the observer wants every step's tracker
+  if (count >= 2 && resolve_variant(s) == DETAG_VARIANT_DENSE && s->n <= 32 && s->y_obs == nullptr) {
+    StepParams p = make_params(s);
+    p.t_noise = static_cast<uint32_t>(s->t + 1);
+    p.steps = count;
+    const int e = detag::launch_step_mma_many(p, s->sm_count, static_cast<cudaStream_t>(stream));
+    if (e != 0) return fail_cuda(s, e, "detag_step_many launch");
+    s->t += count;
+    return DETAG_OK;
+  }
+  for (int i = 0; i < count; ++i) {
+    const int rc = detag_step(s, stream);
+    if (rc != DETAG_OK) return rc;
+  }
+  return DETAG_OK;
+}
+
 int detag_host_staging_bytes(const detag_state* s, int64_t chunk_coords, size_t* bytes) {
   if (!s || !bytes || chunk_coords < 128 || (chunk_coords % 128) != 0) return DETAG_ERR_ARG;
   *bytes = ws_layout(s).total + static_cast<size_t>(2) * 5 * s->n * static_cast<size_t>(chunk_coords) * sizeof(float);

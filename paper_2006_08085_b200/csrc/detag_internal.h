@@ -45,6 +45,7 @@ struct StepParams {
   uint32_t seed_lo, seed_hi;
   uint32_t t_noise;  // step index that enters the noise counter
   int grad_at_start;  // nonzero: the gradient is taken at the model the step started from (Algorithm 2 as printed)
+  int steps;          // consecutive steps in one launch (multi-step kernel only)
   int* status;
 };
 
@@ -61,6 +62,7 @@ int plan_step_csr(StepParams& p, int smem_optin_bytes);  // chooses S; DETAG_ERR
 int launch_step_csr(const StepParams& p, int sm_count, cudaStream_t stream);
 bool dense_variant_available(int n);  // n <= kMaxDenseWorkers and the driver offers tensor-map encoding
 int launch_step_mma(StepParams p, int sm_count, cudaStream_t stream);           // FP64 tensor path, n <= 32
+int launch_step_mma_many(StepParams p, int sm_count, cudaStream_t stream);      // p.steps steps in one launch, n <= 32
 bool band_variant_available(int n, int half_band);  // circulant band kernel: n % 32 == 0, n >= 64, half-band <= 16
 bool dense_window_available(int n);                // the band kernel's dense mode: 32 < n <= 64
 int launch_step_band(StepParams p, const double* band /* null: dense mode */, int sm_count, cudaStream_t stream);

@@ -79,6 +79,9 @@ class Session:
         for _ in range(count):
             B.detag_step(self.state, st)
 
+    def step_many(self, count: int) -> None:
+        B.detag_step_many(self.state, count, self.stream())
+
     def consensus_error(self) -> float:
         return B.detag_consensus_error(self.state, self.stream())
 

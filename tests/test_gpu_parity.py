@@ -230,6 +230,22 @@ def test_misuse_is_reported_not_faulted():
         B.detag_destroy(st)
 
 
+def test_paper_experiment_settings():
+    """The (eta, R) pairs and ring/slack matrices of the paper's own runs, on the synthetic objective: every
+    variant that accepts them, one step per element and a short trajectory.  eta is the paper's tuned value, not
+    the one Algorithm 3 derives from lambda."""
+    from conftest import read_golden
+
+    for row in read_golden("table_detag_hyperparameters.txt"):
+        n, kappa, eta, R = int(row[0]), float(row[1]), float(row[2]), int(row[3])
+        m = inputs.slack_matrix(inputs.metropolis_weights(inputs.ring_graph(n)), kappa)
+        rng = np.random.default_rng(int(1000 * kappa) + n)
+        a, c = _random_objective(rng, n, 1500)
+        x0 = (0.01 * rng.standard_normal((1, 1500))).repeat(n, 0).astype(np.float32)
+        _check_one_step(m, R, eta, 0.05, a, c, x0, 0.1, 17)
+        _check_trajectory(m, R, eta, 0.05, a, c, x0, 0.1, 17, steps=8)
+
+
 # ----------------------------------------------------------------------------- the five configurations
 def _config_case(name, d):
     cfg = inputs.CONFIGS[name]
