@@ -443,11 +443,12 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
         float2 xo, yo, go;
         xo.x = static_cast<float>(cx[t][0]);                              // x' (Algorithm 2's model update)
         xo.y = static_cast<float>(cx[t][1]);
+        const bool row_ok = rb * kR + orow < n;  // dense mode pads n up to 64: padded rows exist on chip only
         const long long off = static_cast<long long>(rb * kR + orow) * p.ld + j;
         // Gradient point: the new model, or (Algorithm 2 as printed) the model before this step.  The old x and g
         // of this tile are still in global memory: its stores are issued after all of its warps are done.
         float2 x_at = xo;
-        if (p.grad_at_start) {
+        if (p.grad_at_start && row_ok) {
           x_at.x = j < p.d ? p.x[off] : 0.f;
           x_at.y = j + 1 < p.d ? p.x[off + 1] : 0.f;
         }
@@ -459,11 +460,11 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
         *reinterpret_cast<float2*>(ob + ooff) = xo;
         *reinterpret_cast<float2*>(ob + kR * kS + ooff) = yo;
         *reinterpret_cast<float2*>(ob + 2 * kR * kS + ooff) = go;
-        if (p.y_obs != nullptr) {  // optional observer: the gossiped tracker y~ = (y~ - g) + g, stored directly
+        if (p.y_obs != nullptr && row_ok) {  // optional observer: the gossiped tracker y~ = (y~ - g) + g, stored directly
           if (j < p.d) p.y_obs[off] = static_cast<float>(cy[t][0] + static_cast<double>(p.g[off]));
           if (j + 1 < p.d) p.y_obs[off + 1] = static_cast<float>(cy[t][1] + static_cast<double>(p.g[off + 1]));
         }
-        if (j >= d_tma) {  // the last d % 4 coordinates: TMA clips stores at 16-byte granularity
+        if (j >= d_tma && row_ok) {  // the last d % 4 coordinates: TMA clips stores at 16-byte granularity
           if (j < p.d) {
             p.x[off] = xo.x;
             p.y[off] = yo.x;

@@ -94,7 +94,8 @@ def _check_trajectory(m, K, eta, alpha, a, c, x0, sigma, seed, steps, j0=0, vari
 
 
 # ----------------------------------------------------------------------------- small and edge cases
-@pytest.mark.parametrize("n,d,K", [(3, 1, 1), (5, 37, 2), (8, 300, 3), (8, 129, 16), (7, 4, 5), (12, 1025, 4)])
+@pytest.mark.parametrize("n,d,K", [(3, 1, 1), (5, 37, 2), (8, 300, 3), (8, 129, 16), (7, 4, 5), (12, 1025, 4),
+                                   (33, 130, 2), (40, 257, 3), (50, 64, 4), (63, 67, 5)])
 def test_small_rings_ragged_sizes(n, d, K):
     rng = np.random.default_rng(n * 1000 + d)
     m = inputs.metropolis_weights(inputs.ring_graph(n))
@@ -181,7 +182,8 @@ def test_noise_matches_the_counter_based_definition():
 
 
 @pytest.mark.parametrize("n,d,K,kind", [(64, 130, 16, "ring"), (96, 67, 5, "ring"), (64, 200, 4, "directed"),
-                                         (128, 64, 8, "two_hop"), (256, 129, 16, "slack")])
+                                         (128, 64, 8, "two_hop"), (256, 129, 16, "slack"), (512, 70, 8, "ring"),
+                                         (1024, 33, 4, "ring")])
 def test_circulant_band_variant(n, d, K, kind):
     """Circulant matrices take the banded-polynomial kernel: symmetric ring, a NON-symmetric circulant (fixes the
     sign of the band offset), a two-hop circulant (bandwidth 2), and a slack ring."""
