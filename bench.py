@@ -34,12 +34,12 @@ BYTES_PER_WC = 32  # read x, y, g, a, c + write x, y, g, float32 each: the fused
 # small case of the same kernel; traffic grows in proportion to n*d).  Keyed by the sha256 prefix of the kernel
 # source the capture was taken on: a changed kernel reports null until it is captured again.
 MEASURED_TRAFFIC = {
-    # cfg5 shape, d = 2,000,000: 1.2854 GB read + 0.7178 GB written / 64 M wc
-    ("step_mma.cu", "dense"): ("996d4601c5b9033f", 31.30),
-    # cfg4 shape, d = 200,000: 1.0270 GB read + 0.5706 GB written / 51.2 M wc (the re-read halo rows come from L2)
-    ("step_band.cu", "ring"): ("ef85fb13d585b2ae", 31.20),
-    # cfg3 shape, d = 500,000: 0.6447 GB read + 0.3369 GB written / 32 M wc
-    ("step_band.cu", "dense"): ("ef85fb13d585b2ae", 30.68),
+    # cfg5 shape, d = 2,000,000: 1.2848 GB read + 0.7180 GB written / 64 M wc
+    ("step_mma.cu", "dense"): ("bfb7c3e6dba76294", 31.29),
+    # cfg4 shape, d = 200,000: 1.0265 GB read + 0.5697 GB written / 51.2 M wc (the re-read halo rows come from L2)
+    ("step_band.cu", "ring"): ("ec846b1e607a1f60", 31.18),
+    # cfg3 shape, d = 500,000: 0.6404 GB read + 0.3374 GB written / 32 M wc
+    ("step_band.cu", "dense"): ("ec846b1e607a1f60", 30.56),
 }
 
 # Float64 multiply-adds per worker-coordinate on the FP64 tensor pipe (both contractions, padded shapes) and that

@@ -18,7 +18,9 @@ namespace detag {
 
 namespace {
 
-template <bool kAtStart>
+// kKs: number of 4-worker input blocks that can be non-zero, ceil(n / 4) rounded up to 2, 4 or 8; the MMAs of the
+// all-zero blocks of the padded P are not issued.
+template <bool kAtStart, int kKs>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 step_mma_many_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
   // No static shared memory in this kernel: the dynamic array starts at the CTA's shared window, whose
@@ -169,7 +171,7 @@ step_mma_many_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
           cx[t][0] = cx[t][1] = 0.0;
         }
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
+        for (int ks = 0; ks < kKs; ++ks) {
           const int src = (4 * ks + kq) * kPitchXY + cl + r;
           const double by = static_cast<double>(sy[src]);
           const double bx = fma(-alpha, by, static_cast<double>(sx[src]));
@@ -264,7 +266,13 @@ int launch_step_mma_many(StepParams p, int sm_count, cudaStream_t stream) {
   if (p.steps < 1 || !make_mma_maps(&maps, p)) return static_cast<int>(cudaErrorInvalidValue);
   p.S = kS;
   p.num_slabs = (p.d + kS - 1) / kS;
-  auto kernel = p.grad_at_start ? step_mma_many_kernel<true> : step_mma_many_kernel<false>;
+  void (*kernel)(const StepParams, const MmaMaps);
+  if (p.n <= 8)
+    kernel = p.grad_at_start ? step_mma_many_kernel<true, 2> : step_mma_many_kernel<false, 2>;
+  else if (p.n <= 16)
+    kernel = p.grad_at_start ? step_mma_many_kernel<true, 4> : step_mma_many_kernel<false, 4>;
+  else
+    kernel = p.grad_at_start ? step_mma_many_kernel<true, 8> : step_mma_many_kernel<false, 8>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(kMmaSmemBytes));
   if (e != cudaSuccess) return static_cast<int>(e);
