@@ -394,12 +394,19 @@ int detag_step_many(detag_state* s, int count, void* stream) {
   if (!s->bound) return fail(s, DETAG_ERR_UNBOUND, "detag_step_many before detag_bind");
   // the fused kernel exists for the dense polynomial with n <= 32; the observer wants every step's tracker
   if (count >= 2 && resolve_variant(s) == DETAG_VARIANT_DENSE && s->n <= 32 && s->y_obs == nullptr) {
-    StepParams p = make_params(s);
-    p.t_noise = static_cast<uint32_t>(s->t + 1);
-    p.steps = count;
-    const int e = detag::launch_step_mma_many(p, s->sm_count, static_cast<cudaStream_t>(stream));
-    if (e != 0) return fail_cuda(s, e, "detag_step_many launch");
-    s->t += count;
+    // A launch is cut off at kMaxFusedSteps so that no thread of the kernel waits on a peer for longer than its
+    // bounded waits allow (a tile of 1024 steps takes some tens of milliseconds; the waits give up after seconds).
+    constexpr int kMaxFusedSteps = 1024;
+    for (int done = 0; done < count;) {
+      const int now = count - done < kMaxFusedSteps ? count - done : kMaxFusedSteps;
+      StepParams p = make_params(s);
+      p.t_noise = static_cast<uint32_t>(s->t + 1);
+      p.steps = now;
+      const int e = detag::launch_step_mma_many(p, s->sm_count, static_cast<cudaStream_t>(stream));
+      if (e != 0) return fail_cuda(s, e, "detag_step_many launch");
+      s->t += now;
+      done += now;
+    }
     return DETAG_OK;
   }
   for (int i = 0; i < count; ++i) {

@@ -27,7 +27,8 @@ def _case(n, d, seed):
     return m, eta, a, c, x0
 
 
-@pytest.mark.parametrize("n,d,K,count", [(8, 4096, 2, 10), (16, 10_003, 4, 7), (32, 20_001, 6, 5), (5, 37, 3, 4), (3, 2, 1, 3)])
+@pytest.mark.parametrize("n,d,K,count", [(8, 4096, 2, 10), (16, 10_003, 4, 7), (32, 20_001, 6, 5), (5, 37, 3, 4), (3, 2, 1, 3),
+                                         (8, 64, 2, 1030)])  # more than one launch's worth of fused steps
 @pytest.mark.parametrize("where", [B.DETAG_GRADIENT_AT_NEW_MODEL, B.DETAG_GRADIENT_AT_PHASE_START])
 def test_fused_steps_equal_single_steps_bit_for_bit(n, d, K, count, where):
     m, eta, a, c, x0 = _case(n, d, n + d)
