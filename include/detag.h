@@ -148,7 +148,7 @@ int detag_get_gradient_point(const detag_state* s, int* where);
 int detag_phase_length(int n, double lambda, double varsigma0_sq, double T, double delta_L, int* R);
 
 /*
- * Initial state of Algorithm 2 as the task fixes it: g = stochastic gradient at the bound x
+ * Initial state of Algorithm 2 (which leaves the tracker's start open): g = stochastic gradient at the bound x
  * (noise of step 0), y = g.  Sets the step counter to 0.  Asynchronous.  Errors: UNBOUND, CUDA.
  */
 int detag_init(detag_state* s, void* stream);

@@ -11,7 +11,7 @@ i.e. ``M[i,j]`` is the paper's ``W_ji`` (Eq. "gossip update" and Algorithm 3).
 State arrays have shape ``[n, m]``: worker i in row i, m coordinates (any coordinate
 subset: the step never mixes coordinates).
 
-Step (order of the operations as the task states them; Algorithm 2 gives the updates):
+Step (gradient evaluated last, at the new model; Algorithm 2 gives the updates):
 
     (a) fold      y   <- y + g_new - g_old                      Algorithm 2, tracker update
     (b) gossip    y   <- AG_K(y) ;  x <- AG_K(x) - alpha*y      Algorithm 2 (AG calls, model update)
