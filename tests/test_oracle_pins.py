@@ -53,6 +53,22 @@ def test_noise_is_standard_normal_and_independent():
     assert abs(np.corrcoef(xi[0] ** 2, xi[1] ** 2)[0, 1]) < 1.5e-2
 
 
+def test_box_muller_radius_and_angle_follow_their_uniforms():
+    """A pair's radius is the chi-square(2) quantile of u_rad and its angle is 2 pi u_ang (library routines, not the
+    oracle's formula): fixes which word feeds which, the 23-bit uniforms and the cos/sin order."""
+    seed, t, n, j0, j1 = 21, 5, 8, 4000, 4300
+    xi = orc.standard_normal_noise(seed, t, n, j0, j1)
+    j = np.arange(j0, j1, dtype=np.uint64)
+    for q in range(n // 4):
+        r = philox4x32_10(j & np.uint64(0xFFFFFFFF), j >> np.uint64(32), np.uint64(q), np.uint64(t), seed, 0)
+        for pair in range(2):
+            first, second = xi[4 * q + 2 * pair], xi[4 * q + 2 * pair + 1]
+            u_rad = ((r[2 * pair] >> np.uint32(9)).astype(np.float64) + 0.5) / 2.0 ** 23
+            u_ang = (r[2 * pair + 1] >> np.uint32(9)).astype(np.float64) / 2.0 ** 23
+            assert np.allclose(first ** 2 + second ** 2, scipy.stats.chi2(2).isf(u_rad), rtol=1e-10)
+            assert np.allclose(np.mod(np.arctan2(second, first), 2 * math.pi), 2 * math.pi * u_ang, atol=1e-9)
+
+
 def test_noise_is_a_pure_function_of_its_counter():
     full = orc.standard_normal_noise(5, 2, 6, 0, 300)
     part = orc.standard_normal_noise(5, 2, 6, 100, 260)
