@@ -32,6 +32,9 @@ constexpr unsigned kMmaSpinLimit = 1u << 20;  // polls before a wait gives up (e
 constexpr unsigned kSuspendHintNs = 2000;
 constexpr size_t kMmaSmemBytes =
     static_cast<size_t>(kMmaStages) * kStageBytes + kWarpGroups * kOutFloats * 4 + kFragBytes + 128;
+// the last 128 bytes hold the mbarriers (full, empty per stage; ready, free per output tile) and the group counters
+static_assert((2 * kMmaStages + 2 * kWarpGroups) * 8 + kWarpGroups * 4 <= 128, "barrier area");
+static_assert(kMmaSmemBytes <= 232448, "shared memory plan");
 
 struct MmaMaps {
   CUtensorMap x, y, g, a, c;  // loads (padded boxes)
