@@ -317,6 +317,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "peak_source": peak_src, "bytes_per_wc": BYTES_PER_WC,
                          "kernel_ms": kernel_ms, "kernel_ms_min": float(per_step.min()),
+                         "kernel_ms_median": float(np.median(per_step)),
                          "frac_of_8TBps_nominal": achieved / 8000.0, "fp64_tensor_pipe": fp64},
             "clocks": clocks,
             "gpu_launches": args.steps,
