@@ -150,11 +150,12 @@ bool dense_ok(const detag_state* s) {
 
 // Host cost model.  The dense product needs n multiply-adds per element and array against the sparse
 // rounds' K*(nnz per row), but keeps its outputs in registers and needs no barriers; it wins for every
-// n it supports.
+// n it supports - except that for 32 < n <= 64 a circulant matrix with a narrow band is cheaper through the
+// band kernel (80 instead of 128 MMAs per tile).
 int resolve_variant(const detag_state* s) {
   if (s->variant_forced != DETAG_VARIANT_AUTO) return s->variant_forced;
+  if (s->n > 32 && band_ok(s)) return DETAG_VARIANT_RING;
   if (dense_ok(s)) return DETAG_VARIANT_DENSE;
-  if (band_ok(s)) return DETAG_VARIANT_RING;
   return DETAG_VARIANT_CSR;
 }
 
