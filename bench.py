@@ -8,6 +8,10 @@ model update, stochastic gradient) over all n workers of the chosen synthetic co
 (launched by torch.distributed.run, one rank per GPU) every rank steps its own coordinate shard of the same
 size; the step has no exchange between coordinates, so there is no data-path collective (weak scaling).
 
+With --gpus N > 1 and no launcher around it (WORLD_SIZE unset) the script starts its own N ranks through
+torch.distributed.run on 127.0.0.1.  `--host-only` (used by the CPU test of that path) makes the ranks meet over
+gloo, exchange the two scalars the real run reduces, and stop before the first CUDA call.
+
 Prints ONE JSON line on rank 0.  `--impl reference` times the float64 CPU oracle on a bounded sample instead.
 """
 from __future__ import annotations
@@ -32,42 +36,50 @@ BYTES_PER_WC = 32  # read x, y, g, a, c + write x, y, g, float32 each: the fused
 
 # DRAM traffic per worker-coordinate (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture on a
 # small case of the same kernel; traffic grows in proportion to n*d).  Keyed by the sha256 prefix of the kernel
-# source the capture was taken on: a changed kernel reports null until it is captured again.
+# sources the capture was taken on: a changed kernel reports null until it is captured again.
+KERNEL_SOURCES = {
+    "mma": ("step_mma.cu", "mma_common.cuh", "pipeline.cuh", "noise.cuh"),
+    "band": ("step_band.cu", "pipeline.cuh", "noise.cuh"),
+    "csr": ("step_csr.cu", "noise.cuh"),
+}
 MEASURED_TRAFFIC = {
-    # cfg5 shape, d = 2,000,000: 1.2848 GB read + 0.7180 GB written / 64 M wc
-    ("step_mma.cu", "dense"): ("bfb7c3e6dba76294", 31.29),
-    # cfg4 shape, d = 200,000: 1.0265 GB read + 0.5697 GB written / 51.2 M wc (the re-read halo rows come from L2)
-    ("step_band.cu", "ring"): ("ec846b1e607a1f60", 31.18),
-    # cfg3 shape, d = 500,000: 0.6404 GB read + 0.3374 GB written / 32 M wc
-    ("step_band.cu", "dense"): ("ec846b1e607a1f60", 30.56),
+    # (kernel, mode): (source digest, bytes per wc)
 }
 
-# Float64 multiply-adds per worker-coordinate on the FP64 tensor pipe (both contractions, padded shapes) and that
+# Float64 multiply-adds per worker-coordinate on the FP64 pipe (both contractions, padded shapes) and that
 # pipe's peak: 64 multiply-adds per clock and SM (measured: 61 with m8n8k4 MMAs from 16 warps) x 148 SMs x max clock.
-FP64_FMA_PER_WC = {("step_mma.cu", "dense"): 64, ("step_band.cu", "ring"): 80, ("step_band.cu", "dense"): 128}
+FP64_FMA_PER_WC = {("mma", "dense"): 64, ("band", "ring"): 80, ("band", "dense"): 128}
 FP64_FMA_PER_CLK_SM = 64
 SM_COUNT = 148
 
 
 def kernel_key(variant: str, n: int):
     if variant == "dense":
-        return ("step_mma.cu", "dense") if n <= 32 else ("step_band.cu", "dense")
+        return ("mma", "dense") if n <= 32 else ("band", "dense")
     if variant == "ring":
-        return ("step_band.cu", "ring")
+        return ("band", "ring")
+    if variant == "csr":
+        return ("csr", "rounds")
     return None
 
 
-def measured_traffic_bytes(variant: str, n: int, wc: int):
+def source_digest(kernel: str) -> str:
     import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES[kernel]:
+        with open(os.path.join(ROOT, "paper_2006_08085_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def measured_traffic_bytes(variant: str, n: int, wc: int):
     key = kernel_key(variant, n)
-    if key is None:
+    if key is None or key not in MEASURED_TRAFFIC:
         return None
     digest, per_wc = MEASURED_TRAFFIC[key]
-    path = os.path.join(ROOT, "paper_2006_08085_b200", "csrc", key[0])
     try:
-        with open(path, "rb") as fh:
-            if hashlib.sha256(fh.read()).hexdigest()[:16] != digest:
-                return None
+        if source_digest(key[0]) != digest:
+            return None
     except OSError:
         return None
     return per_wc * wc
@@ -83,25 +95,67 @@ def measured_peak_gbs():
 
 
 # ------------------------------------------------------------------------------------ oracle timing
-def oracle_throughput(cfg, budget_s: float, sample_d: int, steps: int):
-    """Times the float64 oracle (as it stands, one process) on `sample_d` coordinates; returns a dict."""
+def _oracle_sample(cfg, j0: int, m: int):
+    """The oracle's problem and initial state for coordinates [j0, j0 + m) of a configuration."""
     from oracle import detag_oracle as orc
 
-    sub = cfg.with_d(min(sample_d, cfg.d))
-    m = inputs.gossip_matrix(sub)
-    eta = orc.spectrum(m.to_dense()).eta
-    a, c, x0 = inputs.objective_data(sub)
-    p = orc.Problem(m.row_ptr, m.col_idx, m.vals, sub.K, eta, sub.alpha, a, c, sub.sigma, sub.seed, 0)
-    s = orc.init_state(p, x0)
+    gm = inputs.gossip_matrix(cfg)
+    eta = orc.spectrum(gm.to_dense()).eta
+    a, c, x0 = inputs.objective_data(cfg, j0, j0 + m)
+    p = orc.Problem(gm.row_ptr, gm.col_idx, gm.vals, cfg.K, eta, cfg.alpha, a, c, cfg.sigma, cfg.seed, j0)
+    return orc, p, orc.init_state(p, x0)
+
+
+def oracle_throughput(cfg, budget_s: float, sample_d: int, steps: int):
+    """Times the float64 oracle (as it stands, one process) on `sample_d` coordinates; returns a dict."""
+    m = min(sample_d, cfg.d)
+    orc, p, s = _oracle_sample(cfg, 0, m)
     done, t0 = 0, time.perf_counter()
     while done < steps and (done == 0 or time.perf_counter() - t0 < budget_s):
         s = orc.step(p, s)
         done += 1
     dt = time.perf_counter() - t0
-    return {"value": sub.wc * done / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"{done} steps of {sub.name} on the first {sub.d} of {cfg.d} coordinates "
-                      f"(all {sub.n} workers), {dt:.1f} s, single process",
-            "_ms_per_step": dt / done * 1e3, "_steps": done, "_sample_wc": sub.wc}
+    return {"value": cfg.n * m * done / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{done} steps of {cfg.name} on the first {m} of {cfg.d} coordinates "
+                      f"(all {cfg.n} workers), {dt:.1f} s, single process",
+            "_ms_per_step": dt / done * 1e3, "_steps": done, "_sample_wc": cfg.n * m}
+
+
+def _oracle_worker(job):
+    """One process of the all-cores leg: its own coordinate range, stepped until the time budget is spent."""
+    name, j0, m, budget_s = job
+    cfg = inputs.CONFIGS[name]
+    orc, p, s = _oracle_sample(cfg, j0, m)
+    done, t0 = 0, time.perf_counter()
+    while done == 0 or time.perf_counter() - t0 < budget_s:
+        s = orc.step(p, s)
+        done += 1
+    return done, time.perf_counter() - t0
+
+
+def oracle_throughput_all_cores(cfg, budget_s: float, sample_d: int):
+    """One oracle process per host core on disjoint coordinate ranges (the step never mixes coordinates).
+    The processes are started with `spawn`: a process forked after the first CUDA call would hang."""
+    import multiprocessing as mp
+
+    cores = min(os.cpu_count() or 1, 128)
+    m = max(1, min(sample_d, cfg.d // cores))
+    os.environ.setdefault("OMP_NUM_THREADS", "1")  # one core per process: no nested threading in the children
+    jobs = [(cfg.name, k * m, m, budget_s) for k in range(cores)]
+    with mp.get_context("spawn").Pool(cores) as pool:
+        res = pool.map(_oracle_worker, jobs)
+    value = sum(cfg.n * m * done / dt for done, dt in res)
+    return {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{cores} processes, one per host core, each stepping its own {m} coordinates of {cfg.name} "
+                      f"(all {cfg.n} workers) for {budget_s:.0f} s: {sum(d for d, _ in res)} steps in total"}
+
+
+def cpu_baseline(cfg, budget_s: float):
+    sample_d = max(1024, min(cfg.d, 400_000 // cfg.n))
+    one = oracle_throughput(cfg, budget_s, sample_d, 10 ** 9)
+    out = oracle_throughput_all_cores(cfg, budget_s, sample_d)
+    out["one_core"] = {k: v for k, v in one.items() if not k.startswith("_")}
+    return out
 
 
 def run_reference(args, rank: int) -> None:
@@ -173,6 +227,90 @@ def physical_gpu_index(local_rank: int) -> int:
         except Exception:
             return local_rank
     return local_rank
+
+
+def time_config(name: str, dev, args) -> dict:
+    """Device-resident step time of one configuration at its full size (a short run: 3 warm-up steps, then 20
+    or 200 timed ones), with both roofline fractions.  Inputs are the configuration's own seeded arrays."""
+    import torch
+
+    from paper_2006_08085_b200 import binding as B
+    from paper_2006_08085_b200.session import Session
+
+    cfg = inputs.CONFIGS[name]
+    gm = inputs.gossip_matrix(cfg)
+    ld = (cfg.d + 3) // 4 * 4
+    s = Session(gm, cfg.d, cfg.K, float("nan"), cfg.alpha, None, None, None, cfg.sigma, cfg.seed, ld=ld, device=str(dev))
+    chunk = 1 << 21
+    for j0 in range(0, cfg.d, chunk):  # objective data chunk by chunk: bounded host memory
+        j1 = min(cfg.d, j0 + chunk)
+        a, c, x0 = inputs.objective_data(cfg, j0, j1, threads=min(32, os.cpu_count() or 1))
+        for nm, arr in (("a", a), ("c", c), ("x", x0)):
+            getattr(s, nm)[:, j0:j1].copy_(torch.from_numpy(arr))
+    variant = {1: "csr", 2: "dense", 3: "ring"}.get(B.detag_get_variant(s.state), "other")
+    stream = torch.cuda.current_stream(dev)
+    s.init()
+    steps = 200 if 20 * cfg.wc < 4 * 126e6 else 20
+    for _ in range(3):
+        B.detag_step(s.state, stream)
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        B.detag_step(s.state, stream)
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    s.status()
+    ms = e0.elapsed_time(e1) / steps
+    ce = s.consensus_error()
+    s.close()
+    del s
+    torch.cuda.empty_cache()
+    peak, _ = measured_peak_gbs()
+    achieved = BYTES_PER_WC * cfg.wc / (ms * 1e-3) / 1e9
+    key = kernel_key(variant, cfg.n)
+    out = {"workload": cfg.name, "n": cfg.n, "d": cfg.d, "K": cfg.K, "graph": cfg.graph, "variant": variant,
+           "steps": steps, "ms_per_step": ms, "value": cfg.wc / (ms * 1e-3), "unit": UNIT,
+           "achieved_gbs": achieved, "frac_of_measured_peak": achieved / peak,
+           "frac_of_8TBps_nominal": achieved / 8000.0, "consensus_error_after_run": ce,
+           "l2": "exceeds L2" if 20 * cfg.wc > 4 * 126e6 else "working set fits the 126 MB L2: not an HBM measurement"}
+    if key in FP64_FMA_PER_WC:
+        out["fp64_fma_per_wc"] = FP64_FMA_PER_WC[key]
+        out["fp64_pipe_frac"] = FP64_FMA_PER_WC[key] * out["value"] / (FP64_FMA_PER_CLK_SM * SM_COUNT * 1965e6)
+    return out
+
+
+def run_host_only(args, rank: int, world: int) -> None:
+    """The multi-rank plumbing without a GPU: the ranks meet over gloo, work out their shards and reduce the two
+    scalars the real run reduces (slowest rank's time, sum of the shards' consensus errors)."""
+    import torch.distributed as dist
+
+    from paper_2006_08085_b200 import sharding
+
+    if world > 1:
+        dist.init_process_group("gloo")
+    cfg = inputs.CONFIGS[args.config]
+    offset = sharding.weak_scaling_offset(cfg.d, rank)
+    slowest = sharding.reduce_max(1.0 + rank, dist if world > 1 else None)
+    total = sharding.reduce_sum(float(offset), dist if world > 1 else None)
+    if rank == 0:
+        print(json.dumps({"host_only": True, "n_gpus": world, "slowest": slowest, "offset_sum": total,
+                          "config": {"workload": cfg.name}}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def spawn_ranks(n: int) -> int:
+    """Starts n ranks of this script through torch.distributed.run on the loopback address and waits for them."""
+    import socket
+    import subprocess
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def run_ours(args, rank: int, world: int, local_rank: int) -> None:
@@ -256,6 +394,39 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
                  "ms_per_step": ms, "value": cfg.wc / (ms * 1e-3), "unit": UNIT,
                  "hbm_bytes_per_wc_per_step": BYTES_PER_WC / T if variant == "dense" and cfg.n <= 32 else BYTES_PER_WC}
 
+    # ---- extra: the other step modes on the same buffers (D-PSGD: 24 B/wc; caller-written gradients: 28 B/wc)
+    modes = None
+    if world == 1 and not args.no_modes:
+        modes = {}
+        m_steps = max(3, min(20, args.steps))
+
+        def timed(label, bytes_per_wc):
+            for _ in range(3):
+                B.detag_step(s.state, stream)
+            m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            m0.record(stream)
+            for _ in range(m_steps):
+                B.detag_step(s.state, stream)
+            m1.record(stream)
+            torch.cuda.synchronize(dev)
+            s.status()
+            ms = m0.elapsed_time(m1) / m_steps
+            gbs = bytes_per_wc * cfg.wc / (ms * 1e-3) / 1e9
+            modes[label] = {"ms_per_step": ms, "value": cfg.wc / (ms * 1e-3), "unit": UNIT, "steps": m_steps,
+                            "bytes_per_wc": bytes_per_wc, "achieved_gbs": gbs,
+                            "variant": {1: "csr", 2: "dense", 3: "ring"}.get(B.detag_get_variant(s.state), "other")}
+
+        B.detag_set_algorithm(s.state, B.DETAG_ALGORITHM_DPSGD)
+        timed("dpsgd", 24)
+        B.detag_set_algorithm(s.state, B.DETAG_ALGORITHM_DETAG)
+        g_new = torch.empty_like(s.g)
+        g_new.copy_(s.g)
+        B.detag_set_gradient_source(s.state, B.DETAG_GRADIENT_EXTERNAL, g_new)
+        timed("external_gradient", 28)  # the same gradient array every step: the traffic is what is timed
+        B.detag_set_gradient_source(s.state, B.DETAG_GRADIENT_SYNTHETIC, None)
+        del g_new
+        s.init()  # a clean DeTAG state for the legs below
+
     # ---- end to end through the host-buffer entry point: H2D of x, y, g, a, c and D2H of x, y, g every step
     e2e = None
     if not args.no_e2e:
@@ -292,6 +463,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
                "api": "detag_step_host (page-locked host state; chunked copy/step/copy on two streams)"}
         del staging
 
+    line = None
     if rank == 0:
         peak, peak_src = measured_peak_gbs()
         kernel_ms = float(per_step.mean())
@@ -299,7 +471,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         traffic = measured_traffic_bytes(variant, cfg.n, cfg.wc)
         key = kernel_key(variant, cfg.n)
         fp64, fp64_peak = None, None
-        if key is not None:  # second roofline: the FP64 tensor pipe that carries both contractions
+        if key in FP64_FMA_PER_WC:  # second roofline: the FP64 pipe that carries both contractions
             fma = FP64_FMA_PER_WC[key] * cfg.wc / (kernel_ms * 1e-3)
             fp64_peak = FP64_FMA_PER_CLK_SM * SM_COUNT * (clocks.get("sm_max_mhz") or 1965) * 1e6
             fp64 = {"fma_per_wc": FP64_FMA_PER_WC[key], "achieved_tfma_s": fma / 1e12, "peak_tfma_s": fp64_peak / 1e12,
@@ -327,14 +499,24 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         if e2e is not None:
             line["e2e"] = e2e
         if multi is not None:
-            if key is not None:
+            if fp64_peak is not None:
                 multi["fp64_tensor_pipe_frac"] = FP64_FMA_PER_WC[key] * multi["value"] / fp64_peak
             line["multi_step"] = multi
-        if world == 1 and not args.no_cpu_baseline:
-            r = oracle_throughput(cfg, 20.0, max(1024, min(cfg.d, 400_000 // cfg.n)), 1000)
-            line["cpu_baseline"] = {k: v for k, v in r.items() if not k.startswith("_")}
-        print(json.dumps(line), flush=True)
+        if modes is not None:
+            for v in modes.values():
+                v["frac_of_measured_peak"] = v["achieved_gbs"] / peak
+            line["modes"] = modes
+    # the bench configuration's buffers go before the other configurations are set up
     s.close()
+    del s, host
+    torch.cuda.empty_cache()
+    if rank == 0:
+        if world == 1 and not args.no_per_config:
+            line["per_config"] = [time_config(name, dev, args) for name in sorted(inputs.CONFIGS)
+                                  if name != cfg.name or args.d]
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(inputs.CONFIGS[args.config], 10.0)
+        print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
@@ -354,12 +536,20 @@ def main() -> None:
     ap.add_argument("--multi-launches", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the short runs of the other configurations")
+    ap.add_argument("--no-modes", action="store_true", help="skip the D-PSGD and caller-written-gradient legs")
+    ap.add_argument("--host-only", action="store_true",
+                    help="multi-rank plumbing only (gloo, no CUDA call): what the CPU test of --gpus N runs")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        sys.exit(spawn_ranks(args.gpus))  # no launcher around this process: start the ranks here
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+    elif args.host_only:
+        run_host_only(args, rank, world)
     else:
         run_ours(args, rank, world, local_rank)
 

@@ -68,6 +68,18 @@ enum {
   DETAG_GRADIENT_AT_PHASE_START = 1  /* at x, the model the step started from: Algorithm 2 as printed */
 };
 
+/* Which decentralized algorithm a step runs. */
+enum {
+  DETAG_ALGORITHM_DETAG = 0, /* Algorithm 2 with Algorithm 3 as the gossip (default) */
+  DETAG_ALGORITHM_DPSGD = 1  /* D-PSGD, the paper's main baseline: no gradient tracker */
+};
+
+/* Who evaluates the stochastic gradient. */
+enum {
+  DETAG_GRADIENT_SYNTHETIC = 0, /* the library: g = a o (x - c) + sigma xi of the synthetic objective (default) */
+  DETAG_GRADIENT_EXTERNAL = 1   /* the caller (e.g. back-propagation) writes it into a device array before each step */
+};
+
 /*
  * Spectrum of a symmetric gossip matrix and the accelerated-gossip momentum.
  * Paper: Section "Protocol Layer" (lambda = max(|lambda_2|, |lambda_n|)) and Algorithm 3
@@ -98,7 +110,8 @@ int detag_workspace_bytes(const detag_state* s, size_t* bytes);
 /*
  * Bind the caller's device buffers (see the layout conventions above):
  *   x, y, g : state, read and written by detag_init / detag_step
- *   a, c    : objective data, read only
+ *   a, c    : objective data, read only; both may be NULL when every gradient comes from the caller
+ *             (detag_set_gradient_source), otherwise init and step return DETAG_ERR_UNBOUND
  *   workspace: at least detag_workspace_bytes() bytes, 256-byte aligned; the call fills it with
  *              the graph tables (synchronous copies on the current device).
  * Rebinding is allowed (e.g. to step another coordinate shard with the same graph).
@@ -137,6 +150,36 @@ int detag_get_variant(const detag_state* s, int* variant);
  */
 int detag_set_gradient_point(detag_state* s, int where);
 int detag_get_gradient_point(const detag_state* s, int* where);
+
+/*
+ * D-PSGD (the baseline of the paper's Section "Experiments"; update rule in its Section "Related work":
+ * every worker averages its neighbours' models with the gossip matrix and takes a step along its own
+ * stochastic gradient).  With DETAG_ALGORITHM_DPSGD a step is
+ *     x'  = AG_K(x) - alpha * g          (plain D-PSGD is K = 1, eta = 0: x' = M x - alpha g)
+ *     g'  = a o (x' - c) + sigma * xi    (the gradient the NEXT step uses, evaluated at the new model)
+ * on the same kernels, with one contraction and no tracker: the y buffer is neither read nor written, and
+ * 24 bytes per worker-coordinate cross HBM instead of 32.  detag_init then sets g = gradient at the bound x only.
+ * Synthetic gradient only.  Errors: ARG, UNSUPPORTED (combined with caller-written gradients).
+ */
+int detag_set_algorithm(detag_state* s, int algorithm);
+int detag_get_algorithm(const detag_state* s, int* algorithm);
+
+/*
+ * Caller-written stochastic gradients.  In the paper the gradient oracle of Algorithm 2 (Section "Setting",
+ * oracle class; the line of Algorithm 2 that spends the query budget) is back-propagation on a mini-batch, not
+ * a formula.  With DETAG_GRADIENT_EXTERNAL the library evaluates no gradient: before detag_init and before every
+ * detag_step the caller writes the stochastic gradient at the CURRENT model x into g_new (device, [n][ld]
+ * float32, 16-byte aligned, caller-owned, must stay valid), and a step is Algorithm 2 without the query:
+ *     y   = y + g_new - g                tracker update (g = the gradient folded by the previous step)
+ *     y'  = AG_K(y) ;  x' = AG_K(x) - alpha * y'
+ *     g   = g_new                        the library keeps the folded gradient for the next update
+ * so here the y buffer holds the gossiped tracker itself (not the early-folded one of the default mode), and
+ * 28 bytes per worker-coordinate cross HBM.  detag_init sets y = g = g_new (the first update is then the
+ * identity).  a, c, the noise settings and the gradient point are not used.  detag_step_many accepts count = 1
+ * only; detag_step_host is not offered.  DETAG_GRADIENT_SYNTHETIC switches back (g_new is ignored).
+ * Errors: ARG (unknown source, null or misaligned g_new), UNSUPPORTED (combined with D-PSGD).
+ */
+int detag_set_gradient_source(detag_state* s, int source, const float* g_new);
 
 /*
  * Phase length of Theorem 3: R = max(1/2 ln n, 1/2 ln(varsigma0_sq * T / delta_L)) / sqrt(1 - lambda),
@@ -225,8 +268,35 @@ int detag_consensus_error_static(int n, int64_t d, int64_t ld, const float* x, v
 int detag_get_step(const detag_state* s, int64_t* t);
 int detag_set_step(detag_state* s, int64_t t);
 
-/* Waits for `stream`, then returns the device status word: DETAG_OK or DETAG_ERR_TIMEOUT. */
+/*
+ * Waits for `stream`, then reads the device status words - the one in the bound workspace and, if
+ * detag_step_host has run since the last clean detag_status, the one at the head of its staging area
+ * (which must therefore still be allocated) - and returns DETAG_OK, DETAG_ERR_TIMEOUT (a bounded
+ * device-side wait gave up; the state arrays are then not to be trusted) or DETAG_ERR_CUDA.  A state that
+ * has only ever stepped host-resident needs no detag_bind for this call.  The words are sticky: detag_bind
+ * clears the workspace's, a staging area's is cleared when detag_step_host first uses it.
+ * Errors: UNBOUND (neither bound nor stepped host-resident), CUDA, TIMEOUT.
+ */
 int detag_status(detag_state* s, void* stream);
+
+/*
+ * Failure-detection self tests.  The paper has no counterpart (its algorithm is synchronous and assumes
+ * no failures); these exist so that the bounded waits of the kernels, their wind-down and DETAG_ERR_TIMEOUT
+ * can be exercised without faulting, trapping or hanging the GPU.
+ *
+ * detag_debug_inject_stall: from now on the loading thread of every CTA of the tensor-path step kernels stops
+ * issuing loads after `after_tiles` tiles, and every device-side wait gives up after `poll_limit` polls
+ * (16 .. 2^20; a poll suspends for at most about two microseconds).  The CTAs' waiters then time out one
+ * after the other, set the status word and return; the launch ends normally and detag_status reports
+ * DETAG_ERR_TIMEOUT.  The state arrays are left partly updated.  after_tiles < 0 restores normal operation
+ * (no stall, default limit).  Host only.  Errors: ARG.
+ *
+ * detag_debug_expire_wait: launches one thread that waits, through the same bounded wait, on a barrier that
+ * nothing ever arrives at, with a limit of `polls` polls (1 .. 2^20); it gives up, sets the workspace's status
+ * word and returns.  Asynchronous.  Errors: ARG, UNBOUND, CUDA.
+ */
+int detag_debug_inject_stall(detag_state* s, int64_t after_tiles, uint32_t poll_limit);
+int detag_debug_expire_wait(detag_state* s, uint32_t polls, void* stream);
 
 /* Text of the last error on this state ("" if none).  Owned by the state. */
 const char* detag_last_error(const detag_state* s);

@@ -230,6 +230,39 @@ def run_as_printed(p: Problem, x0: np.ndarray, phases: int, observe=None) -> Pha
     return s
 
 
+# --------------------------------------------------------------------------------------
+# D-PSGD, the paper's main baseline (Section "Related work"; baselines of Section "Experiments")
+# --------------------------------------------------------------------------------------
+class DpsgdState(NamedTuple):
+    x: np.ndarray
+    g: np.ndarray  # stochastic gradient at the current x
+    t: int  # number of completed steps
+
+
+def init_dpsgd_state(p: Problem, x0: np.ndarray) -> DpsgdState:
+    x = np.array(x0, dtype=np.float64, copy=True)
+    return DpsgdState(x, stochastic_gradient(p, x, 0), 0)
+
+
+def dpsgd_step(p: Problem, s: DpsgdState) -> DpsgdState:
+    """Every worker averages its neighbours' models with the gossip matrix and steps along its own stochastic
+    gradient taken at its own current model: x' = AG_K(x) - alpha * g(x).  Plain D-PSGD is K = 1, eta = 0, where
+    AG_K is one gossip step, x'_i = sum_j W_ji x_j - alpha g_i.  No tracker."""
+    x = accelerated_gossip(s.x, p.row_ptr, p.col_idx, p.vals, p.K, p.eta) - p.alpha * s.g
+    return DpsgdState(x, stochastic_gradient(p, x, s.t + 1), s.t + 1)
+
+
+def run_dpsgd(p: Problem, x0: np.ndarray, steps: int, observe=None) -> DpsgdState:
+    s = init_dpsgd_state(p, x0)
+    if observe is not None:
+        observe(s)
+    for _ in range(steps):
+        s = dpsgd_step(p, s)
+        if observe is not None:
+            observe(s)
+    return s
+
+
 def phase_length(n: int, lam: float, varsigma0_sq: float, T: float, delta_L: float) -> int:
     """Theorem 3's phase length R = max(1/2 ln n, 1/2 ln(varsigma_0^2 T / (Delta L))) / sqrt(1 - lambda),
     rounded up to a whole number of gossip rounds (at least one)."""

@@ -35,6 +35,12 @@ DETAG_VARIANT_RING = 3
 DETAG_GRADIENT_AT_NEW_MODEL = 0
 DETAG_GRADIENT_AT_PHASE_START = 1
 
+DETAG_ALGORITHM_DETAG = 0
+DETAG_ALGORITHM_DPSGD = 1
+
+DETAG_GRADIENT_SYNTHETIC = 0
+DETAG_GRADIENT_EXTERNAL = 1
+
 _ERR_NAMES = {
     -1: "DETAG_ERR_ARG", -2: "DETAG_ERR_CSR", -3: "DETAG_ERR_NOT_STOCHASTIC", -4: "DETAG_ERR_NOT_SYMMETRIC",
     -5: "DETAG_ERR_UNSUPPORTED", -6: "DETAG_ERR_UNBOUND", -7: "DETAG_ERR_CUDA", -8: "DETAG_ERR_TIMEOUT",
@@ -57,6 +63,11 @@ SIGNATURES = {
     "detag_get_variant": (ctypes.c_int, [_P, ctypes.POINTER(ctypes.c_int)]),
     "detag_set_gradient_point": (ctypes.c_int, [_P, ctypes.c_int]),
     "detag_get_gradient_point": (ctypes.c_int, [_P, ctypes.POINTER(ctypes.c_int)]),
+    "detag_set_algorithm": (ctypes.c_int, [_P, ctypes.c_int]),
+    "detag_get_algorithm": (ctypes.c_int, [_P, ctypes.POINTER(ctypes.c_int)]),
+    "detag_set_gradient_source": (ctypes.c_int, [_P, ctypes.c_int, _P]),
+    "detag_debug_inject_stall": (ctypes.c_int, [_P, ctypes.c_int64, ctypes.c_uint32]),
+    "detag_debug_expire_wait": (ctypes.c_int, [_P, ctypes.c_uint32, _P]),
     "detag_phase_length": (ctypes.c_int, [ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_double,
                                           ctypes.c_double, ctypes.POINTER(ctypes.c_int)]),
     "detag_init": (ctypes.c_int, [_P, _P]),
@@ -185,6 +196,29 @@ def detag_get_gradient_point(state) -> int:
     out = ctypes.c_int(0)
     _check(lib().detag_get_gradient_point(state, ctypes.byref(out)), "detag_get_gradient_point", state)
     return int(out.value)
+
+
+def detag_set_algorithm(state, algorithm: int) -> None:
+    _check(lib().detag_set_algorithm(state, int(algorithm)), "detag_set_algorithm", state)
+
+
+def detag_get_algorithm(state) -> int:
+    out = ctypes.c_int(0)
+    _check(lib().detag_get_algorithm(state, ctypes.byref(out)), "detag_get_algorithm", state)
+    return int(out.value)
+
+
+def detag_set_gradient_source(state, source: int, g_new=None) -> None:
+    """g_new: device tensor [n][ld] float32 the caller writes the newest gradient into (external source only)."""
+    _check(lib().detag_set_gradient_source(state, int(source), _dev_ptr(g_new)), "detag_set_gradient_source", state)
+
+
+def detag_debug_inject_stall(state, after_tiles: int, poll_limit: int = 2048) -> None:
+    _check(lib().detag_debug_inject_stall(state, int(after_tiles), int(poll_limit)), "detag_debug_inject_stall", state)
+
+
+def detag_debug_expire_wait(state, polls: int, stream=None) -> None:
+    _check(lib().detag_debug_expire_wait(state, int(polls), _stream_handle(stream)), "detag_debug_expire_wait", state)
 
 
 def detag_phase_length(n: int, lam: float, varsigma0_sq: float = 0.0, T: float = 0.0, delta_L: float = 1.0) -> int:

@@ -2,8 +2,12 @@
 // (used for the initial state) and the consensus-error reduction.
 #include <cuda_runtime.h>
 
+#include <mutex>
+#include <vector>
+
 #include "detag_internal.h"
 #include "noise.cuh"
+#include "pipeline.cuh"
 
 namespace detag {
 
@@ -34,9 +38,34 @@ __global__ void __launch_bounds__(kAuxThreads) init_gradient_kernel(const StepPa
                              sigma * static_cast<double>(xi[w]));
         const float gf = static_cast<float>(g);
         p.g[off] = gf;
-        p.y[off] = gf;
+        if (p.mode != kModeDpsgd) p.y[off] = gf;  // D-PSGD keeps no tracker
       }
     }
+  }
+}
+
+// Caller-written gradients: the initial state is y_0 = g_old = the caller's gradient at x_0, so that the first
+// tracker update of Algorithm 2 (y + g_new - g_old with g_new = g_old) changes nothing.
+__global__ void __launch_bounds__(kAuxThreads) init_external_kernel(const StepParams p) {
+  const long long items = static_cast<long long>(p.n) * p.d;
+  for (long long it = blockIdx.x * static_cast<long long>(kAuxThreads) + threadIdx.x; it < items;
+       it += static_cast<long long>(gridDim.x) * kAuxThreads) {
+    const long long i = it / p.d, j = it - i * p.d;
+    const long long off = i * p.ld + j;
+    const float gv = p.g_ext[off];
+    p.g[off] = gv;
+    p.y[off] = gv;
+  }
+}
+
+// Failure-detection self test: one thread waits, through the kernels' own bounded wait, on a barrier that nobody
+// ever arrives at.  After `polls` polls the wait gives up, the status word is set and the kernel returns normally.
+__global__ void expire_wait_kernel(int* status, unsigned polls) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    bar_init(&bar, 1);
+    fence_barrier_init();
+    if (!bar_wait(&bar, 0, polls)) atomicExch(status, 1);
   }
 }
 
@@ -100,6 +129,45 @@ int launch_init_gradient(const StepParams& p, int sm_count, cudaStream_t stream)
   if (grid > cap) grid = cap;
   init_gradient_kernel<<<static_cast<unsigned>(grid), kAuxThreads, 0, stream>>>(p);
   return static_cast<int>(cudaGetLastError());
+}
+
+int launch_init_external(const StepParams& p, int sm_count, cudaStream_t stream) {
+  const long long items = static_cast<long long>(p.n) * p.d;
+  if (items <= 0) return 0;
+  long long grid = (items + kAuxThreads - 1) / kAuxThreads;
+  const long long cap = static_cast<long long>(sm_count) * 16;
+  if (grid > cap) grid = cap;
+  init_external_kernel<<<static_cast<unsigned>(grid), kAuxThreads, 0, stream>>>(p);
+  return static_cast<int>(cudaGetLastError());
+}
+
+int launch_expire_wait(int* status, unsigned polls, cudaStream_t stream) {
+  expire_wait_kernel<<<1, 32, 0, stream>>>(status, polls);
+  return static_cast<int>(cudaGetLastError());
+}
+
+int ensure_dynamic_smem(const void* kernel, int bytes) {
+  struct Entry {
+    const void* kernel;
+    int device, bytes;
+  };
+  static std::mutex mu;
+  static std::vector<Entry> done;  // the largest size configured so far per kernel and device
+  int device = 0;
+  cudaError_t e = cudaGetDevice(&device);
+  if (e != cudaSuccess) return static_cast<int>(e);
+  std::lock_guard<std::mutex> lock(mu);
+  Entry* hit = nullptr;
+  for (auto& en : done)
+    if (en.kernel == kernel && en.device == device) hit = &en;
+  if (hit != nullptr && hit->bytes >= bytes) return 0;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return static_cast<int>(e);
+  if (hit != nullptr)
+    hit->bytes = bytes;
+  else
+    done.push_back(Entry{kernel, device, bytes});
+  return 0;
 }
 
 int launch_consensus_error(const StepParams& p, double* partials, double* result, int sm_count,

@@ -116,6 +116,11 @@ bool band_ok(const detag_state* s) {
   return s->circulant && s->d <= 0x7fffffffLL && detag::band_variant_available(s->n, s->half_band);
 }
 
+int step_mode(const detag_state* s) {
+  if (s->algorithm == DETAG_ALGORITHM_DPSGD) return detag::kModeDpsgd;
+  return s->gradient_source == DETAG_GRADIENT_EXTERNAL ? detag::kModeExternal : detag::kModeDetag;
+}
+
 StepParams make_params(const detag_state* s) {
   StepParams p{};
   p.n = s->n;
@@ -141,6 +146,10 @@ StepParams make_params(const detag_state* s) {
   p.seed_hi = static_cast<uint32_t>(s->seed >> 32);
   p.status = s->d_status;
   p.grad_at_start = s->gradient_point == DETAG_GRADIENT_AT_PHASE_START ? 1 : 0;
+  p.mode = step_mode(s);
+  p.g_ext = s->g_ext;
+  p.spin_limit = s->spin_limit;
+  p.stall_after = s->stall_after;
   return p;
 }
 
@@ -151,9 +160,16 @@ bool dense_ok(const detag_state* s) {
 // Host cost model.  The dense product needs n multiply-adds per element and array against the sparse
 // rounds' K*(nnz per row), but keeps its outputs in registers and needs no barriers; it wins for every
 // n it supports - except that for 32 < n <= 64 a circulant matrix with a narrow band is cheaper through the
-// band kernel (80 instead of 128 MMAs per tile).
+// band kernel (80 instead of 128 MMAs per tile).  Caller-written gradients and D-PSGD run on the dense
+// kernel for n <= 32 and on the generic rounds kernel otherwise.
+bool variant_runs_mode(const detag_state* s, int variant) {
+  if (step_mode(s) == detag::kModeDetag) return true;
+  return variant == DETAG_VARIANT_CSR || (variant == DETAG_VARIANT_DENSE && s->n <= 32);
+}
+
 int resolve_variant(const detag_state* s) {
   if (s->variant_forced != DETAG_VARIANT_AUTO) return s->variant_forced;
+  if (step_mode(s) != detag::kModeDetag) return (s->n <= 32 && dense_ok(s)) ? DETAG_VARIANT_DENSE : DETAG_VARIANT_CSR;
   if (s->n > 32 && band_ok(s)) return DETAG_VARIANT_RING;
   if (dense_ok(s)) return DETAG_VARIANT_DENSE;
   return DETAG_VARIANT_CSR;
@@ -171,17 +187,62 @@ int query_device(detag_state* s) {
   return DETAG_OK;
 }
 
+// Kernel families that take tensor maps.
+enum { kFamilyMma = 1, kFamilyBand = 2 };
+
+// Tensor maps for the buffers in `p`: built on first use, then found again by buffer addresses and sizes
+// (detag_step always hits; detag_step_host cycles through its two chunk slots and the ragged last chunk).
+const detag::TensorMapSet* maps_for(detag_state* s, int family, const StepParams& p) {
+  const void* slot_a = p.mode == detag::kModeExternal ? static_cast<const void*>(p.g_ext) : p.a;
+  const void* key[5] = {p.x, p.mode == detag::kModeDpsgd ? nullptr : p.y, p.g, slot_a,
+                        p.mode == detag::kModeExternal ? nullptr : p.c};
+  for (auto& en : s->map_cache) {
+    if (en.family == family && en.d == p.d && en.ld == p.ld && std::memcmp(en.ptr, key, sizeof key) == 0)
+      return &en.maps;
+  }
+  constexpr size_t kEntries = 6;
+  detag_state::MapEntry* slot;
+  if (s->map_cache.size() < kEntries) {
+    s->map_cache.emplace_back();
+    slot = &s->map_cache.back();
+  } else {
+    slot = &s->map_cache[s->map_next];
+    s->map_next = (s->map_next + 1) % kEntries;
+  }
+  detag_state::MapEntry& en = *slot;
+  en.family = 0;  // invalid until built
+  const bool ok = family == kFamilyMma ? detag::build_maps_mma(p, &en.maps) : detag::build_maps_band(p, &en.maps);
+  if (!ok) return nullptr;
+  en.family = family;
+  en.d = p.d;
+  en.ld = p.ld;
+  std::memcpy(en.ptr, key, sizeof key);
+  return &en.maps;
+}
+
 // Picks the kernel variant, plans it for the sizes in `p` and launches it.
 int launch_step(detag_state* s, StepParams& p, cudaStream_t stream) {
   int e = 0;
-  switch (resolve_variant(s)) {
+  const int variant = resolve_variant(s);
+  if (!variant_runs_mode(s, variant))
+    return fail(s, DETAG_ERR_UNSUPPORTED,
+                "this kernel variant runs the DeTAG step with the synthetic gradient only; use AUTO or CSR");
+  if (p.mode != detag::kModeExternal && (!p.a || !p.c))
+    return fail(s, DETAG_ERR_UNBOUND, "the synthetic gradient needs the objective arrays a and c");
+  if (p.mode == detag::kModeExternal && !p.g_ext)
+    return fail(s, DETAG_ERR_UNBOUND, "caller-written gradients selected but no gradient array given");
+  switch (variant) {
     case DETAG_VARIANT_DENSE:
-      e = p.n <= 32 ? detag::launch_step_mma(p, s->sm_count, stream)
-                    : detag::launch_step_band(p, nullptr, s->sm_count, stream);
+    case DETAG_VARIANT_RING: {
+      const bool mma = variant == DETAG_VARIANT_DENSE && p.n <= 32;
+      const detag::TensorMapSet* maps = maps_for(s, mma ? kFamilyMma : kFamilyBand, p);
+      if (!maps) return fail(s, DETAG_ERR_CUDA, "tensor map encoding failed");
+      if (mma)
+        e = detag::launch_step_mma(p, *maps, s->sm_count, stream);
+      else
+        e = detag::launch_step_band(p, *maps, variant == DETAG_VARIANT_RING ? s->band : nullptr, s->sm_count, stream);
       break;
-    case DETAG_VARIANT_RING:
-      e = detag::launch_step_band(p, s->band, s->sm_count, stream);
-      break;
+    }
     case DETAG_VARIANT_CSR:
     default: {
       const int rc = detag::plan_step_csr(p, s->smem_optin);
@@ -239,6 +300,7 @@ int detag_create(detag_state** out, int n, int64_t d, const int32_t* row_ptr, co
   s->vals.assign(vals, vals + nnz);
   if (n <= detag::kMaxDenseWorkers) gossip_polynomial(s, s->poly);
   analyse_circulant(s);
+  s->map_cache.reserve(8);
   *out = s;
   return DETAG_OK;
 }
@@ -252,9 +314,9 @@ int detag_workspace_bytes(const detag_state* s, size_t* bytes) {
 int detag_bind(detag_state* s, int64_t ld, float* x, float* y, float* g, const float* a, const float* c,
                void* workspace, size_t workspace_bytes) {
   if (!s) return DETAG_ERR_ARG;
-  if (!x || !y || !g || !a || !c || !workspace) return fail(s, DETAG_ERR_ARG, "detag_bind: null buffer");
+  if (!x || !y || !g || !workspace) return fail(s, DETAG_ERR_ARG, "detag_bind: null buffer");
   if (ld < s->d || (ld & 3) != 0) return fail(s, DETAG_ERR_ARG, "detag_bind: ld must be >= d and a multiple of 4");
-  if (!aligned16(x) || !aligned16(y) || !aligned16(g) || !aligned16(a) || !aligned16(c))
+  if (!aligned16(x) || !aligned16(y) || !aligned16(g) || !aligned16(a) || !aligned16(c))  // NULL counts as aligned
     return fail(s, DETAG_ERR_ARG, "detag_bind: state arrays must be 16-byte aligned");
   if ((reinterpret_cast<uintptr_t>(workspace) % detag::kWsAlign) != 0)
     return fail(s, DETAG_ERR_ARG, "detag_bind: workspace must be 256-byte aligned");
@@ -355,6 +417,62 @@ int detag_get_gradient_point(const detag_state* s, int* where) {
   return DETAG_OK;
 }
 
+int detag_set_algorithm(detag_state* s, int algorithm) {
+  if (!s) return DETAG_ERR_ARG;
+  if (algorithm != DETAG_ALGORITHM_DETAG && algorithm != DETAG_ALGORITHM_DPSGD)
+    return fail(s, DETAG_ERR_ARG, "detag_set_algorithm: unknown value");
+  if (algorithm == DETAG_ALGORITHM_DPSGD && s->gradient_source == DETAG_GRADIENT_EXTERNAL)
+    return fail(s, DETAG_ERR_UNSUPPORTED, "detag_set_algorithm: D-PSGD runs with the synthetic gradient only");
+  s->algorithm = algorithm;
+  return DETAG_OK;
+}
+
+int detag_get_algorithm(const detag_state* s, int* algorithm) {
+  if (!s || !algorithm) return DETAG_ERR_ARG;
+  *algorithm = s->algorithm;
+  return DETAG_OK;
+}
+
+int detag_set_gradient_source(detag_state* s, int source, const float* g_new) {
+  if (!s) return DETAG_ERR_ARG;
+  if (source == DETAG_GRADIENT_SYNTHETIC) {
+    s->gradient_source = source;
+    s->g_ext = nullptr;
+    return DETAG_OK;
+  }
+  if (source != DETAG_GRADIENT_EXTERNAL) return fail(s, DETAG_ERR_ARG, "detag_set_gradient_source: unknown value");
+  if (!g_new || !aligned16(g_new))
+    return fail(s, DETAG_ERR_ARG, "detag_set_gradient_source: the gradient array must be non-null and 16-byte aligned");
+  if (s->algorithm == DETAG_ALGORITHM_DPSGD)
+    return fail(s, DETAG_ERR_UNSUPPORTED, "detag_set_gradient_source: D-PSGD runs with the synthetic gradient only");
+  s->gradient_source = source;
+  s->g_ext = g_new;
+  return DETAG_OK;
+}
+
+int detag_debug_inject_stall(detag_state* s, int64_t after_tiles, uint32_t poll_limit) {
+  if (!s) return DETAG_ERR_ARG;
+  if (after_tiles < 0) {  // back to normal
+    s->stall_after = -1;
+    s->spin_limit = 1u << 20;
+    return DETAG_OK;
+  }
+  if (poll_limit < 16 || poll_limit > (1u << 20))
+    return fail(s, DETAG_ERR_ARG, "detag_debug_inject_stall: poll limit outside [16, 2^20]");
+  s->stall_after = after_tiles;
+  s->spin_limit = poll_limit;
+  return DETAG_OK;
+}
+
+int detag_debug_expire_wait(detag_state* s, uint32_t polls, void* stream) {
+  if (!s) return DETAG_ERR_ARG;
+  if (!s->bound) return fail(s, DETAG_ERR_UNBOUND, "detag_debug_expire_wait before detag_bind");
+  if (polls < 1 || polls > (1u << 20)) return fail(s, DETAG_ERR_ARG, "detag_debug_expire_wait: polls outside [1, 2^20]");
+  const int e = detag::launch_expire_wait(s->d_status, polls, static_cast<cudaStream_t>(stream));
+  if (e != 0) return fail_cuda(s, e, "detag_debug_expire_wait launch");
+  return DETAG_OK;
+}
+
 int detag_phase_length(int n, double lambda, double varsigma0_sq, double T, double delta_L, int* R) {
   if (!R || n < 1 || !(lambda >= 0.0) || !(lambda < 1.0)) return DETAG_ERR_ARG;
   double num = 0.5 * std::log(static_cast<double>(n));
@@ -372,7 +490,14 @@ int detag_init(detag_state* s, void* stream) {
   if (!s->bound) return fail(s, DETAG_ERR_UNBOUND, "detag_init before detag_bind");
   StepParams p = make_params(s);
   p.t_noise = 0;
-  const int e = detag::launch_init_gradient(p, s->sm_count, static_cast<cudaStream_t>(stream));
+  int e;
+  if (p.mode == detag::kModeExternal) {
+    if (!p.g_ext) return fail(s, DETAG_ERR_UNBOUND, "caller-written gradients selected but no gradient array given");
+    e = detag::launch_init_external(p, s->sm_count, static_cast<cudaStream_t>(stream));
+  } else {
+    if (!p.a || !p.c) return fail(s, DETAG_ERR_UNBOUND, "the synthetic gradient needs the objective arrays a and c");
+    e = detag::launch_init_gradient(p, s->sm_count, static_cast<cudaStream_t>(stream));
+  }
   if (e != 0) return fail_cuda(s, e, "detag_init launch");
   s->t = 0;
   return DETAG_OK;
@@ -393,8 +518,11 @@ int detag_step_many(detag_state* s, int count, void* stream) {
   if (!s) return DETAG_ERR_ARG;
   if (count < 1) return fail(s, DETAG_ERR_ARG, "detag_step_many: count must be at least 1");
   if (!s->bound) return fail(s, DETAG_ERR_UNBOUND, "detag_step_many before detag_bind");
+  if (count >= 2 && step_mode(s) == detag::kModeExternal)
+    return fail(s, DETAG_ERR_ARG, "detag_step_many: caller-written gradients need one call per step");
   // the fused kernel exists for the dense polynomial with n <= 32; the observer wants every step's tracker
-  if (count >= 2 && resolve_variant(s) == DETAG_VARIANT_DENSE && s->n <= 32 && s->y_obs == nullptr) {
+  if (count >= 2 && resolve_variant(s) == DETAG_VARIANT_DENSE && s->n <= 32 && s->y_obs == nullptr &&
+      step_mode(s) == detag::kModeDetag) {
     // A launch is cut off at kMaxFusedSteps so that no thread of the kernel waits on a peer for longer than its
     // bounded waits allow (a tile of 1024 steps takes some tens of milliseconds; the waits give up after seconds).
     constexpr int kMaxFusedSteps = 1024;
@@ -403,7 +531,10 @@ int detag_step_many(detag_state* s, int count, void* stream) {
       StepParams p = make_params(s);
       p.t_noise = static_cast<uint32_t>(s->t + 1);
       p.steps = now;
-      const int e = detag::launch_step_mma_many(p, s->sm_count, static_cast<cudaStream_t>(stream));
+      if (!p.a || !p.c) return fail(s, DETAG_ERR_UNBOUND, "the synthetic gradient needs the objective arrays a and c");
+      const detag::TensorMapSet* maps = maps_for(s, kFamilyMma, p);
+      if (!maps) return fail(s, DETAG_ERR_CUDA, "tensor map encoding failed");
+      const int e = detag::launch_step_mma_many(p, *maps, s->sm_count, static_cast<cudaStream_t>(stream));
       if (e != 0) return fail_cuda(s, e, "detag_step_many launch");
       s->t += now;
       done += now;
@@ -427,6 +558,8 @@ int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* 
                     void* staging, size_t staging_bytes, void* stream) {
   if (!s) return DETAG_ERR_ARG;
   if (!x || !y || !g || !a || !c || !staging) return fail(s, DETAG_ERR_ARG, "detag_step_host: null buffer");
+  if (step_mode(s) == detag::kModeExternal)
+    return fail(s, DETAG_ERR_UNSUPPORTED, "detag_step_host: caller-written gradients are not offered on host-resident state");
   if (ld_host < s->d) return fail(s, DETAG_ERR_ARG, "detag_step_host: ld_host < d");
   if ((reinterpret_cast<uintptr_t>(staging) % detag::kWsAlign) != 0)
     return fail(s, DETAG_ERR_ARG, "detag_step_host: staging must be 256-byte aligned");
@@ -449,8 +582,11 @@ int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* 
 
   cudaStream_t user = static_cast<cudaStream_t>(stream);
   unsigned char* base = static_cast<unsigned char*>(staging);
-  // graph tables at the head of the staging area, ordered on the caller's stream
-  e = cudaMemsetAsync(base, 0, detag::kWsAlign, user);
+  // Graph tables at the head of the staging area, ordered on the caller's stream.  The status word there is
+  // cleared when a staging area is first used, not on every call: a time-out stays visible to detag_status.
+  int* status_word = reinterpret_cast<int*>(base + l.status);
+  if (s->d_status_host != status_word) e = cudaMemsetAsync(base, 0, detag::kWsAlign, user);
+  s->d_status_host = status_word;
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(base + l.row_ptr, s->row_ptr.data(), s->row_ptr.size() * sizeof(int32_t),
                         cudaMemcpyHostToDevice, user);
@@ -470,7 +606,7 @@ int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* 
   p.col_idx = reinterpret_cast<int32_t*>(base + l.col_idx);
   p.vals = reinterpret_cast<double*>(base + l.vals);
   p.poly = s->poly.empty() ? nullptr : reinterpret_cast<double*>(base + l.poly);
-  p.status = reinterpret_cast<int*>(base + l.status);
+  p.status = status_word;
   p.y_obs = nullptr;
   p.t_noise = static_cast<uint32_t>(s->t + 1);
   p.ld = chunk;
@@ -537,13 +673,18 @@ int detag_set_step(detag_state* s, int64_t t) {
 
 int detag_status(detag_state* s, void* stream) {
   if (!s) return DETAG_ERR_ARG;
-  if (!s->bound) return fail(s, DETAG_ERR_UNBOUND, "detag_status before detag_bind");
-  int word = 0;
+  if (!s->bound && !s->d_status_host) return fail(s, DETAG_ERR_UNBOUND, "detag_status before detag_bind or detag_step_host");
+  int word[2] = {0, 0};
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  cudaError_t e = cudaMemcpyAsync(&word, s->d_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+  cudaError_t e = cudaSuccess;
+  if (s->bound) e = cudaMemcpyAsync(&word[0], s->d_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess && s->d_status_host)
+    e = cudaMemcpyAsync(&word[1], s->d_status_host, sizeof(int), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) return fail_cuda(s, e, "detag_status");
-  if (word != 0) return fail(s, DETAG_ERR_TIMEOUT, "a device-side wait gave up");
+  if (word[0] == 2 || word[1] == 2) return fail(s, DETAG_ERR_CUDA, "a kernel found its shared memory misaligned");
+  if (word[0] != 0 || word[1] != 0) return fail(s, DETAG_ERR_TIMEOUT, "a device-side wait gave up");
+  s->d_status_host = nullptr;  // read and clean: the staging area is not referred to again until the next host step
   return DETAG_OK;
 }
 

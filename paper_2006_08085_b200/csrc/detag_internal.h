@@ -46,7 +46,22 @@ struct StepParams {
   uint32_t t_noise;  // step index that enters the noise counter
   int grad_at_start;  // nonzero: the gradient is taken at the model the step started from (Algorithm 2 as printed)
   int steps;          // consecutive steps in one launch (multi-step kernel only)
+  int mode;           // kModeDetag, kModeExternal or kModeDpsgd
+  const float* g_ext; // kModeExternal: the caller's newest stochastic gradient, [n][ld]
+  unsigned spin_limit;    // polls after which a device-side wait gives up
+  long long stall_after;  // failure-detection self test: a CTA's producer stops loading after this many tiles (< 0: off)
   int* status;
+};
+
+// What a step computes (the `mode` of StepParams)
+constexpr int kModeDetag = 0;     // DeTAG with the library's own synthetic gradient (y holds the folded tracker)
+constexpr int kModeExternal = 1;  // DeTAG with caller-written gradients: fold, gossip, model update; no gradient evaluation
+constexpr int kModeDpsgd = 2;     // D-PSGD: x' = AG_K(x) - alpha g, g' = synthetic gradient at x'; no tracker
+
+// Room for the tensor maps of one launch (eight 128-byte CUtensorMap objects), built once per set of bound
+// buffers and kept in the state.
+struct alignas(64) TensorMapSet {
+  unsigned char bytes[8 * 128];
 };
 
 // host helpers (spectral.cpp)
@@ -61,12 +76,21 @@ int launch_init_gradient(const StepParams& p, int sm_count, cudaStream_t stream)
 int plan_step_csr(StepParams& p, int smem_optin_bytes);  // chooses S; DETAG_ERR_UNSUPPORTED if nothing fits
 int launch_step_csr(const StepParams& p, int sm_count, cudaStream_t stream);
 bool dense_variant_available(int n);  // n <= kMaxDenseWorkers and the driver offers tensor-map encoding
-int launch_step_mma(StepParams p, int sm_count, cudaStream_t stream);           // FP64 tensor path, n <= 32
-int launch_step_mma_many(StepParams p, int sm_count, cudaStream_t stream);      // p.steps steps in one launch, n <= 32
+// Tensor-path kernels: build_* fills the tensor maps for the buffers in `p` (false: the driver refused one);
+// launch_* takes the maps built for exactly those buffers.
+bool build_maps_mma(const StepParams& p, TensorMapSet* maps);
+int launch_step_mma(StepParams p, const TensorMapSet& maps, int sm_count, cudaStream_t stream);       // n <= 32
+int launch_step_mma_many(StepParams p, const TensorMapSet& maps, int sm_count, cudaStream_t stream);  // p.steps steps
 bool band_variant_available(int n, int half_band);  // circulant band kernel: n % 32 == 0, n >= 64, half-band <= 16
 bool dense_window_available(int n);                // the band kernel's dense mode: 32 < n <= 64
-int launch_step_band(StepParams p, const double* band /* null: dense mode */, int sm_count, cudaStream_t stream);
+bool build_maps_band(const StepParams& p, TensorMapSet* maps);
+int launch_step_band(StepParams p, const TensorMapSet& maps, const double* band /* null: dense mode */, int sm_count,
+                     cudaStream_t stream);
 int launch_consensus_error(const StepParams& p, double* partials, double* result, int sm_count, cudaStream_t stream);
+int launch_init_external(const StepParams& p, int sm_count, cudaStream_t stream);  // y = g = g_ext
+int launch_expire_wait(int* status, unsigned polls, cudaStream_t stream);          // a wait nobody ends (self test)
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device; returns a cudaError_t value.
+int ensure_dynamic_smem(const void* kernel, int bytes);
 
 }  // namespace detag
 
@@ -83,6 +107,11 @@ struct detag_state {
   double band[33] = {0};     // p(delta) at index delta + 16, valid when circulant and half_band <= 16
   int variant_forced = DETAG_VARIANT_AUTO;
   int gradient_point = DETAG_GRADIENT_AT_NEW_MODEL;
+  int algorithm = DETAG_ALGORITHM_DETAG;
+  int gradient_source = DETAG_GRADIENT_SYNTHETIC;
+  const float* g_ext = nullptr;
+  unsigned spin_limit = 1u << 20;
+  long long stall_after = -1;
 
   bool bound = false;
   long long ld = 0;
@@ -92,6 +121,7 @@ struct detag_state {
   void* ws = nullptr;
   size_t ws_bytes = 0;
   int* d_status = nullptr;
+  int* d_status_host = nullptr;  // status word of the staging area the last detag_step_host used
   double* d_result = nullptr;
   int32_t* d_row_ptr = nullptr;
   int32_t* d_col_idx = nullptr;
@@ -107,6 +137,16 @@ struct detag_state {
   // host-resident stepping: two internal streams and their events, created on first use
   cudaStream_t host_stream[2] = {nullptr, nullptr};
   struct CUevent_st* host_event[3] = {nullptr, nullptr, nullptr};
+
+  // tensor maps of the launches seen so far, keyed by kernel family and buffers (a few entries, round robin)
+  struct MapEntry {
+    int family = 0;
+    const void* ptr[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    long long d = 0, ld = 0;
+    detag::TensorMapSet maps;
+  };
+  std::vector<MapEntry> map_cache;
+  size_t map_next = 0;
 
   int device = -1;
   int sm_count = 0;

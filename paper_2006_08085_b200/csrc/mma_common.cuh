@@ -1,5 +1,5 @@
 // Pieces shared by the dense-polynomial kernels for n <= 32 (step_mma.cu, step_mma_many.cu): tile geometry, the
-// shared-memory plan, mbarrier / TMA / FP64-MMA wrappers and the tensor maps with their host-side set-up.
+// shared-memory plan, the set-up, producer and storing roles of the persistent CTA, and the tensor maps.
 #ifndef DETAG_MMA_COMMON_CUH
 #define DETAG_MMA_COMMON_CUH
 
@@ -8,6 +8,7 @@
 
 #include "detag_internal.h"
 #include "noise.cuh"
+#include "pipeline.cuh"
 #include "tma.cuh"
 
 namespace detag {
@@ -28,94 +29,144 @@ constexpr int kProducerWarp = kConsumerWarps, kStoreWarp = kConsumerWarps + 1;
 constexpr int kMmaThreads = (kConsumerWarps + 2) * 32;
 constexpr int kOutFloats = 3 * kN * kS;       // x', y', g' tiles of one slab, dense rows
 constexpr int kFragBytes = 32 * 32 * 8;       // P in fragment order
-constexpr unsigned kMmaSpinLimit = 1u << 20;  // polls before a wait gives up (each may suspend ~kSuspendHintNs)
-constexpr unsigned kSuspendHintNs = 2000;
 constexpr size_t kMmaSmemBytes =
     static_cast<size_t>(kMmaStages) * kStageBytes + kWarpGroups * kOutFloats * 4 + kFragBytes + 128;
 // the last 128 bytes hold the mbarriers (full, empty per stage; ready, free per output tile) and the group counters
 static_assert((2 * kMmaStages + 2 * kWarpGroups) * 8 + kWarpGroups * 4 <= 128, "barrier area");
 static_assert(kMmaSmemBytes <= 232448, "shared memory plan");
 
+// Loads (padded boxes): x, y, g and two more arrays - the objective data a, c, or (caller-written gradients) the
+// newest gradient in the `a` slot.  Stores (exact slab width): x', y', g'.
 struct MmaMaps {
-  CUtensorMap x, y, g, a, c;  // loads (padded boxes)
-  CUtensorMap xs, ys, gs;     // stores (exact slab width)
+  CUtensorMap x, y, g, a, c;
+  CUtensorMap xs, ys, gs;
+};
+static_assert(sizeof(MmaMaps) <= sizeof(TensorMapSet), "tensor map storage");
+
+// Pointers into the CTA's dynamic shared memory.
+struct MmaShared {
+  float* stage_mem;     // [stage][x | y | g | a | c]
+  float* out_mem;       // [group][x', y', g'][32][kS]
+  double* frag;         // P in fragment order: [t][ks][lane]
+  uint64_t* full;       // [stage]: the stage's loads have landed
+  uint64_t* empty;      // [stage]: the group's warps no longer read the stage
+  uint64_t* out_ready;  // [group]: the group's 8 warps have written their outputs
+  uint64_t* out_free;   // [group]: the stores have finished reading the tile
+  unsigned* seen;       // [group]: 1 + last slab index whose data the group saw
 };
 
-__device__ __forceinline__ uint32_t s_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ bool bar_wait(uint64_t* bar, unsigned parity) {
-  const uint32_t addr = s_addr(bar);
-  for (unsigned spin = 0; spin < kMmaSpinLimit; ++spin) {
-    unsigned done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(addr), "r"(parity), "r"(kSuspendHintNs)
-        : "memory");
-    if (done) return true;
-  }
-  return false;
-}
-
-// Monotonic progress counter in shared memory (release/acquire at CTA scope), bounded wait.
-__device__ __forceinline__ void count_publish(unsigned* counter, unsigned value) {
-  asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(s_addr(counter)), "r"(value) : "memory");
-}
-
-__device__ __forceinline__ bool count_wait(const unsigned* counter, unsigned at_least) {
-  const uint32_t addr = s_addr(counter);
-  for (unsigned spin = 0; spin < kMmaSpinLimit; ++spin) {
-    unsigned v;
-    asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-    if (v >= at_least) return true;
-    __nanosleep(100);
-  }
-  return false;
-}
-
-__device__ __forceinline__ void bar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_addr(bar)) : "memory");
-}
-
-__device__ __forceinline__ void bar_init(uint64_t* bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_addr(bar)), "r"(count));
-}
-
-__device__ __forceinline__ void tile_load(float* dst, const CUtensorMap* map, int col, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-          s_addr(dst)),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(col), "r"(0), "r"(s_addr(bar))
-      : "memory");
-}
-
-__device__ __forceinline__ void tile_store(const CUtensorMap* map, int col, const float* src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
-                   reinterpret_cast<uint64_t>(map)),
-               "r"(col), "r"(0), "r"(s_addr(src))
-               : "memory");
-}
-
-__device__ __forceinline__ void dmma(double (&c)[2], double a, double b) {
-  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-               : "+d"(c[0]), "+d"(c[1])
-               : "d"(a), "d"(b));
-}
-
-// Tensor maps over the bound arrays; false when the driver refuses one.
-inline bool make_mma_maps(MmaMaps* maps, const StepParams& p) {
-  if (!make_map(&maps->x, p.x, p.n, p.d, p.ld, kN, kPitchXY) || !make_map(&maps->y, p.y, p.n, p.d, p.ld, kN, kPitchXY) ||
-      !make_map(&maps->g, p.g, p.n, p.d, p.ld, kN, kPitchE) || !make_map(&maps->a, p.a, p.n, p.d, p.ld, kN, kPitchE) ||
-      !make_map(&maps->c, p.c, p.n, p.d, p.ld, kN, kPitchE))
+// Carves up the shared memory, writes P in fragment order and initialises the barriers.  Returns false (and
+// sets status 2) when the shared window is not 128-byte aligned, which the TMA tiles need.  All threads call it.
+__device__ __forceinline__ bool mma_setup(const StepParams& p, unsigned char* smem_raw, MmaShared& sm) {
+  sm.stage_mem = reinterpret_cast<float*>(smem_raw);
+  sm.out_mem = sm.stage_mem + kMmaStages * kStageFloats;
+  sm.frag = reinterpret_cast<double*>(sm.out_mem + kWarpGroups * kOutFloats);
+  sm.full = reinterpret_cast<uint64_t*>(sm.frag + 32 * 32);
+  sm.empty = sm.full + kMmaStages;
+  sm.out_ready = sm.empty + kMmaStages;
+  sm.out_free = sm.out_ready + kWarpGroups;
+  sm.seen = reinterpret_cast<unsigned*>(sm.out_free + kWarpGroups);
+  if ((s_addr(smem_raw) & 127u) != 0) {
+    if (threadIdx.x == 0) atomicExch(p.status, 2);
     return false;
-  const long long d_tma = p.d & ~3LL;  // the stores' tensor ends on a 16-byte boundary (see the kernels' tails)
-  if (d_tma > 0 && (!make_map(&maps->xs, p.x, p.n, d_tma, p.ld, kN, kS) || !make_map(&maps->ys, p.y, p.n, d_tma, p.ld, kN, kS) ||
-                    !make_map(&maps->gs, p.g, p.n, d_tma, p.ld, kN, kS)))
-    return false;
-  if (d_tma == 0) maps->xs = maps->ys = maps->gs = maps->x;  // never used: every slab lies beyond column 0
+  }
+  const int tid = threadIdx.x, n = p.n;
+  // block (t, ks), lane (r, kq) holds P[4r + t][4ks + kq]
+  for (int e = tid; e < 32 * 32; e += kMmaThreads) {
+    const int l = e & 31, ks = (e >> 5) & 7, t = e >> 8;
+    const int i = 4 * (l >> 2) + t, j = 4 * ks + (l & 3);
+    sm.frag[e] = (i < n && j < n) ? p.poly[static_cast<size_t>(i) * n + j] : 0.0;
+  }
+  if (tid == 0) {
+    for (int g = 0; g < kWarpGroups; ++g) sm.seen[g] = 0;
+    for (int s = 0; s < kMmaStages; ++s) {
+      bar_init(&sm.full[s], 1);
+      bar_init(&sm.empty[s], kGroupWarps);
+    }
+    for (int g = 0; g < kWarpGroups; ++g) {
+      bar_init(&sm.out_ready[g], kGroupWarps);
+      bar_init(&sm.out_free[g], 1);
+    }
+    fence_barrier_init();
+  }
+  fence_async_shared();
+  __syncthreads();
   return true;
+}
+
+// Producer role (one thread): keeps kMmaStages slabs in flight.  kMode selects which arrays a stage holds.
+template <int kMode>
+__device__ __forceinline__ void mma_producer(const StepParams& p, const MmaMaps& maps, const MmaShared& sm) {
+  constexpr unsigned kBytes = static_cast<unsigned>(kStageBytes) -
+                              (kMode == kModeDpsgd ? kN * kPitchXY * 4u : 0u) -   // no tracker
+                              (kMode == kModeExternal ? kN * kPitchE * 4u : 0u);  // no objective data
+  const long long first = blockIdx.x, stride = gridDim.x;
+  long long issued = 0;
+  bool ok = true;
+  for (long long slab = first; slab < p.num_slabs; slab += stride, ++issued) {
+    if (p.stall_after >= 0 && issued >= p.stall_after) return;  // self test: the loads stop, every waiter times out
+    const int s = static_cast<int>(issued % kMmaStages);
+    if (issued >= kMmaStages) ok = bar_wait(&sm.empty[s], ((issued / kMmaStages) - 1) & 1, p.spin_limit);
+    if (!ok) break;
+    float* st = sm.stage_mem + static_cast<size_t>(s) * kStageFloats;
+    const int col = static_cast<int>(slab * kS);
+    bar_expect_tx(&sm.full[s], kBytes);
+    tile_load(st, &maps.x, col, 0, &sm.full[s]);
+    if (kMode != kModeDpsgd) tile_load(st + kN * kPitchXY, &maps.y, col, 0, &sm.full[s]);
+    float* se = st + 2 * kN * kPitchXY;
+    tile_load(se, &maps.g, col, 0, &sm.full[s]);
+    tile_load(se + kN * kPitchE, &maps.a, col, 0, &sm.full[s]);
+    if (kMode != kModeExternal) tile_load(se + 2 * kN * kPitchE, &maps.c, col, 0, &sm.full[s]);
+  }
+  if (!ok) {
+    atomicExch(p.status, 1);
+    for (long long back = 1; back <= kMmaStages && back <= issued; ++back) {  // drain copies still in flight (bounded)
+      const long long k = issued - back;
+      bar_wait(&sm.full[k % kMmaStages], (k / kMmaStages) & 1, p.spin_limit);
+    }
+  }
+}
+
+// Storing role (one thread): each finished output tile goes out with one TMA tile store per array.
+template <int kMode>
+__device__ __forceinline__ void mma_storer(const StepParams& p, const MmaMaps& maps, const MmaShared& sm) {
+  const long long first = blockIdx.x, stride = gridDim.x;
+  long long k = 0;
+  for (long long slab = first; slab < p.num_slabs; slab += stride, ++k) {
+    const int g = static_cast<int>(k % kWarpGroups);
+    if (!bar_wait(&sm.out_ready[g], (k / kWarpGroups) & 1, p.spin_limit)) {
+      atomicExch(p.status, 1);
+      break;
+    }
+    const float* ob = sm.out_mem + g * kOutFloats;
+    const int col = static_cast<int>(slab * kS);
+    if (col < (p.d & ~3LL)) {
+      tile_store(&maps.xs, col, 0, ob);
+      if (kMode != kModeDpsgd) tile_store(&maps.ys, col, 0, ob + kN * kS);
+      tile_store(&maps.gs, col, 0, ob + 2 * kN * kS);
+    }
+    store_commit();
+    store_wait_read();  // the tile may be overwritten now
+    bar_arrive(&sm.out_free[g]);
+  }
+  store_wait_all();  // all global writes done before the CTA leaves
+}
+
+// Consumer side: waits until slab k (stage s) of this CTA has landed.  Lane 0 polls, the warp gets the verdict.
+__device__ __forceinline__ bool mma_wait_slab(const StepParams& p, const MmaShared& sm, long long k, int group,
+                                              int tile, int lane) {
+  bool ok = true;
+  if (lane == 0) {
+    const int s = static_cast<int>(k % kMmaStages);
+    // The stage last held slab k - kMmaStages, which belongs to the other group when the stage count is odd.
+    // A parity wait must not start before that phase has completed (it could not tell the two apart), and
+    // it costs nothing to make sure: this slab cannot have been loaded before that one was consumed.
+    if (kMmaStages % kWarpGroups != 0 && k >= kMmaStages)
+      ok = count_wait(&sm.seen[(k - kMmaStages) % kWarpGroups], static_cast<unsigned>(k - kMmaStages + 1), p.spin_limit);
+    if (ok) ok = bar_wait(&sm.full[s], (k / kMmaStages) & 1, p.spin_limit);
+    if (ok && tile == 0) count_publish(&sm.seen[group], static_cast<unsigned>(k + 1));
+  }
+  return __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
 }
 
 }  // namespace

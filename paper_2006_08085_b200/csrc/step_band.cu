@@ -43,6 +43,7 @@
 
 #include "detag_internal.h"
 #include "noise.cuh"
+#include "pipeline.cuh"
 #include "tma.cuh"
 
 namespace detag {
@@ -67,8 +68,6 @@ constexpr int kThreads = (kConsumerWarps + 3) * 32;
 constexpr int kSideFloats = 2 * kHalo * kPitchXY;  // rows 0..15 of x and y, kept for the slab's last row block
 constexpr int kOutFloats = 3 * kR * kS;
 constexpr int kBandSteps = 10;     // 4-row window steps that meet an 8-row output block: (2*16 + 8) / 4
-constexpr unsigned kSpinLimit = 1u << 20;
-constexpr unsigned kSuspendHintNs = 2000;
 constexpr size_t kSmemBytes =
     static_cast<size_t>(kStages) * kStageBytes + 2 * kSideFloats * 4 + kWarpGroups * kOutFloats * 4 + 128;  // + barriers, counters
 constexpr int kDenseFragBytes = 2 * (kW / 4) * 4 * 32 * 8;  // dense mode: [row block][window step][t][lane] doubles
@@ -80,72 +79,11 @@ struct BandMaps {
   CUtensorMap xs, ys, gs;      // stores, 32-row boxes of width kS
 };
 
+static_assert(sizeof(BandMaps) <= sizeof(TensorMapSet), "tensor map storage");
+
 struct BandCoef {
   double p[2 * kHalo + 1];  // p[delta + kHalo] = P[i][(i + delta) mod n]
 };
-
-__device__ __forceinline__ uint32_t s_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ bool bar_wait(uint64_t* bar, unsigned parity) {
-  const uint32_t addr = s_addr(bar);
-  for (unsigned spin = 0; spin < kSpinLimit; ++spin) {
-    unsigned done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(addr), "r"(parity), "r"(kSuspendHintNs)
-        : "memory");
-    if (done) return true;
-  }
-  return false;
-}
-
-// Monotonic progress counter in this CTA's shared memory (release/acquire at CTA scope), bounded wait.
-__device__ __forceinline__ void count_publish(unsigned* counter, unsigned value) {
-  asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(s_addr(counter)), "r"(value) : "memory");
-}
-
-__device__ __forceinline__ bool count_wait(const unsigned* counter, unsigned at_least) {
-  const uint32_t addr = s_addr(counter);
-  for (unsigned spin = 0; spin < kSpinLimit; ++spin) {
-    unsigned v;
-    asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-    if (v >= at_least) return true;
-    __nanosleep(100);
-  }
-  return false;
-}
-
-__device__ __forceinline__ void bar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_addr(bar)) : "memory");
-}
-
-__device__ __forceinline__ void bar_init(uint64_t* bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_addr(bar)), "r"(count));
-}
-
-__device__ __forceinline__ void tile_load(float* dst, const CUtensorMap* map, int col, int row, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-          s_addr(dst)),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(col), "r"(row), "r"(s_addr(bar))
-      : "memory");
-}
-
-__device__ __forceinline__ void tile_store(const CUtensorMap* map, int col, int row, const float* src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
-                   reinterpret_cast<uint64_t>(map)),
-               "r"(col), "r"(row), "r"(s_addr(src))
-               : "memory");
-}
-
-__device__ __forceinline__ void dmma(double (&c)[2], double a, double b) {
-  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-               : "+d"(c[0]), "+d"(c[1])
-               : "d"(a), "d"(b));
-}
 
 // 4 x 4 transpose over the four lanes {lane ^ 0, 4, 8, 12} (lane bits 2 and 3): lane with index q = (lane >> 2) & 3
 // gives row q = v[0..3] and receives column q.
@@ -202,9 +140,9 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
       bar_init(&out_ready[g], kGroupWarps);
       bar_init(&out_free[g], 1);
     }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_barrier_init();
   }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  fence_async_shared();
   __syncthreads();
 
   // this CTA takes slabs blockIdx.x, blockIdx.x + gridDim.x, ...; tile k is row block k % row_blocks of its
@@ -217,7 +155,7 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
     if (lane == 0) {
       for (long long k = 0; k < num_tiles; ++k) {
         const int s = static_cast<int>(k % kStages);
-        if (!bar_wait(&full[s], (k / kStages) & 1)) {
+        if (!bar_wait(&full[s], (k / kStages) & 1, p.spin_limit)) {
           atomicExch(p.status, 1);
           break;
         }
@@ -232,8 +170,9 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
       long long issued = 0;
       bool ok = true;
       for (; issued < num_tiles; ++issued) {
+        if (p.stall_after >= 0 && issued >= p.stall_after) return;  // self test: the loads stop, every waiter times out
         const int s = static_cast<int>(issued % kStages);
-        if (issued >= kStages) ok = bar_wait(&empty[s], ((issued / kStages) - 1) & 1);
+        if (issued >= kStages) ok = bar_wait(&empty[s], ((issued / kStages) - 1) & 1, p.spin_limit);
         if (!ok) break;
         const long long slab_no = issued / row_blocks;
         const int rb = static_cast<int>(issued % row_blocks);
@@ -244,8 +183,7 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
         // the last block's final window piece (rows 0..15) is not loaded: it comes from the side buffer
         const unsigned bytes = static_cast<unsigned>(kStageBytes) - (last ? 2u * 16 * kPitchXY * 4 : 0u) +
                                (!kDense && rb == 0 ? static_cast<unsigned>(kSideFloats) * 4 : 0u);
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_addr(&full[s])), "r"(bytes)
-                     : "memory");
+        bar_expect_tx(&full[s], bytes);
 #pragma unroll
         for (int q = 0; q < kW / 16; ++q) {  // the window wraps around the ring in 16-row pieces
           if (last && q == kW / 16 - 1) continue;
@@ -273,7 +211,7 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
         atomicExch(p.status, 1);
         for (long long back = 1; back <= kStages && back <= issued; ++back) {  // drain copies still in flight (bounded)
           const long long k = issued - back;
-          bar_wait(&full[k % kStages], (k / kStages) & 1);
+          bar_wait(&full[k % kStages], (k / kStages) & 1, p.spin_limit);
         }
       }
     }
@@ -283,14 +221,14 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
     if (lane == 0) {
       for (long long k = 0; k < num_tiles; ++k) {
         const int g = static_cast<int>(k % kWarpGroups);
-        if (!bar_wait(&out_ready[g], (k / kWarpGroups) & 1)) {
+        if (!bar_wait(&out_ready[g], (k / kWarpGroups) & 1, p.spin_limit)) {
           atomicExch(p.status, 1);
           break;
         }
         const long long slab_no = k / row_blocks;
         const int rb = static_cast<int>(k % row_blocks);
         // in-place update: the next block's window (it contains this block's last rows) must have landed
-        if (rb + 1 < row_blocks && !count_wait(landed, static_cast<unsigned>(k + 2))) {
+        if (rb + 1 < row_blocks && !count_wait(landed, static_cast<unsigned>(k + 2), p.spin_limit)) {
           atomicExch(p.status, 1);
           break;
         }
@@ -301,11 +239,11 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
           tile_store(&maps.ys, col, rb * kR, ob + kR * kS);
           tile_store(&maps.gs, col, rb * kR, ob + 2 * kR * kS);
         }
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        store_commit();
+        store_wait_read();
         bar_arrive(&out_free[g]);
       }
-      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+      store_wait_all();
     }
     return;
   }
@@ -343,8 +281,8 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
       // with an odd stage count the stage last served the other group: a parity wait must not start before
       // that phase has completed (it could not tell the two apart); the counter says when it has
       if (kStages % kWarpGroups != 0 && k >= kStages)
-        ok = count_wait(&seen[(k - kStages) % kWarpGroups], static_cast<unsigned>(k - kStages + 1));
-      if (ok) ok = bar_wait(&full[s], (k / kStages) & 1);
+        ok = count_wait(&seen[(k - kStages) % kWarpGroups], static_cast<unsigned>(k - kStages + 1), p.spin_limit);
+      if (ok) ok = bar_wait(&full[s], (k / kStages) & 1, p.spin_limit);
       if (ok && mtile == 0) count_publish(&seen[group], static_cast<unsigned>(k + 1));
     }
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -410,10 +348,13 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
     __syncwarp();
     if (lane == 0) {
       bar_arrive(&empty[s]);  // stage no longer read by this warp
-      if (use > 0) ok = bar_wait(&out_free[group], (use - 1) & 1);  // previous tile of this group stored
-      // the d % 4 tail columns are stored directly (not by the storing thread): same in-place rule for them
-      if (ok && j0 + kS > d_tma && p.d != d_tma && rb + 1 < row_blocks)
-        ok = count_wait(landed, static_cast<unsigned>(k + 2));
+      if (use > 0) ok = bar_wait(&out_free[group], (use - 1) & 1, p.spin_limit);  // previous tile of this group stored
+      // The d % 4 tail columns are stored directly (not by the storing thread): same in-place rule for them.  The
+      // window of the previous block holds this block's first rows as well, and two stages' loads may complete out
+      // of order, so the slab's last block (which has no next window to wait for) waits until every tile up to
+      // its own has landed.
+      if (ok && j0 + kS > d_tma && p.d != d_tma)
+        ok = count_wait(landed, static_cast<unsigned>(k + (rb + 1 < row_blocks ? 2 : 1)), p.spin_limit);
     }
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     if (!ok) {
@@ -478,7 +419,7 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
         }
       }
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // outputs visible to the TMA store
+    fence_async_shared();  // outputs visible to the TMA store
     __syncwarp();
     if (lane == 0) bar_arrive(&out_ready[group]);
   }
@@ -494,31 +435,36 @@ bool dense_window_available(int n) { return n > kR && n <= kW && encode_tiled_fn
 
 bool dense_variant_available(int n) { return n >= 1 && n <= kMaxDenseWorkers && encode_tiled_fn() != nullptr; }
 
-// band == nullptr: dense mode (32 < n <= 64, p.poly holds P_K(M)); otherwise the circulant band of 2*16+1 entries,
-// p(delta) at index delta + 16.
-int launch_step_band(StepParams p, const double* band, int sm_count, cudaStream_t stream) {
-  BandMaps maps;
-  BandCoef coef;
-  const bool dense = band == nullptr;
-  for (int k = 0; k < 2 * kHalo + 1; ++k) coef.p[k] = dense ? 0.0 : band[k];
+bool build_maps_band(const StepParams& p, TensorMapSet* out) {
+  BandMaps& maps = *reinterpret_cast<BandMaps*>(out->bytes);
   const long long d_tma = p.d & ~3LL;
   if (!make_map(&maps.x16, p.x, p.n, p.d, p.ld, 16, kPitchXY) || !make_map(&maps.y16, p.y, p.n, p.d, p.ld, 16, kPitchXY) ||
       !make_map(&maps.g16, p.g, p.n, p.d, p.ld, 16, kPitchE) || !make_map(&maps.a16, p.a, p.n, p.d, p.ld, 16, kPitchE) ||
       !make_map(&maps.c16, p.c, p.n, p.d, p.ld, 16, kPitchE))
-    return static_cast<int>(cudaErrorInvalidValue);
+    return false;
   if (d_tma > 0 && (!make_map(&maps.xs, p.x, p.n, d_tma, p.ld, kR, kS) || !make_map(&maps.ys, p.y, p.n, d_tma, p.ld, kR, kS) ||
                     !make_map(&maps.gs, p.g, p.n, d_tma, p.ld, kR, kS)))
-    return static_cast<int>(cudaErrorInvalidValue);
+    return false;
   if (d_tma == 0) maps.xs = maps.ys = maps.gs = maps.x16;  // never used
+  return true;
+}
+
+// band == nullptr: dense mode (32 < n <= 64, p.poly holds P_K(M)); otherwise the circulant band of 2*16+1 entries,
+// p(delta) at index delta + 16.
+int launch_step_band(StepParams p, const TensorMapSet& maps, const double* band, int sm_count, cudaStream_t stream) {
+  if (p.mode != kModeDetag) return static_cast<int>(cudaErrorInvalidValue);
+  BandCoef coef;
+  const bool dense = band == nullptr;
+  for (int k = 0; k < 2 * kHalo + 1; ++k) coef.p[k] = dense ? 0.0 : band[k];
   p.S = kS;
   p.num_slabs = (p.d + kS - 1) / kS;
   auto kernel = dense ? step_band_kernel<true> : step_band_kernel<false>;
   const size_t smem = kSmemBytes + (dense ? kDenseFragBytes : 0);
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-  if (e != cudaSuccess) return static_cast<int>(e);
+  const int e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), static_cast<int>(smem));
+  if (e != 0) return e;
   const long long grid = p.num_slabs < sm_count ? p.num_slabs : sm_count;
   if (grid <= 0) return 0;
-  kernel<<<static_cast<unsigned>(grid), kThreads, smem, stream>>>(p, maps, coef);
+  kernel<<<static_cast<unsigned>(grid), kThreads, smem, stream>>>(p, *reinterpret_cast<const BandMaps*>(maps.bytes), coef);
   return static_cast<int>(cudaGetLastError());
 }
 

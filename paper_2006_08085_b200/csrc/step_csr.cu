@@ -12,6 +12,10 @@
 //      float32 value of g' that is stored, so that the stored tracker telescopes exactly
 //      against the stored gradients.
 // All on-chip arithmetic is float64; each result is rounded once when it is stored.
+//
+// Modes: with caller-written gradients step 1 also applies Algorithm 2's tracker update, y + g_new - g_old, and
+// step 3 stores the gossiped tracker and copies g_new over g_old instead of evaluating a gradient; in D-PSGD
+// mode only the model is gossiped and x' = x~ - alpha g.
 #include <cuda_runtime.h>
 
 #include "detag_internal.h"
@@ -60,7 +64,9 @@ __global__ void __launch_bounds__(kCsrThreads) step_csr_kernel(const StepParams 
       if (col < width) {
         const long long off = static_cast<long long>(i) * p.ld + j0 + col;
         vx = static_cast<double>(p.x[off]);
-        vy = static_cast<double>(p.y[off]);
+        if (p.mode != kModeDpsgd) vy = static_cast<double>(p.y[off]);
+        if (p.mode == kModeExternal)  // Algorithm 2's tracker update with the caller's newest gradient
+          vy += static_cast<double>(p.g_ext[off]) - static_cast<double>(p.g[off]);
       }
       cur_x[e] = vx;
       prv_x[e] = vx;
@@ -82,7 +88,7 @@ __global__ void __launch_bounds__(kCsrThreads) step_csr_kernel(const StepParams 
           ay = fma(w, cy[src], ay);
         }
         px[e] = fma(one_plus_eta, ax, -eta * px[e]);
-        py[e] = fma(one_plus_eta, ay, -eta * py[e]);
+        py[e] = fma(one_plus_eta, ay, -eta * py[e]);  // D-PSGD: an all-zero slab, never stored
       }
       __syncthreads();
       double* t;
@@ -96,13 +102,30 @@ __global__ void __launch_bounds__(kCsrThreads) step_csr_kernel(const StepParams 
       if (col >= width) continue;
       const long long j = j0 + col;
       float xi[4] = {0.f, 0.f, 0.f, 0.f};
-      if (sigma != 0.0)
+      if (sigma != 0.0 && p.mode != kModeExternal)
         normal_quad(p.seed_lo, p.seed_hi, static_cast<unsigned long long>(p.coord_offset + j), q, p.t_noise, xi);
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
         const int i = 4 * q + w;
         if (i < n) {
           const long long off = static_cast<long long>(i) * p.ld + j;
+          if (p.mode == kModeExternal) {
+            const double y_gossip = cy[i * S + col];
+            p.x[off] = static_cast<float>(cx[i * S + col] - alpha * y_gossip);
+            p.y[off] = static_cast<float>(y_gossip);
+            p.g[off] = p.g_ext[off];  // the gradient just folded is the next step's g_old
+            if (p.y_obs != nullptr) p.y_obs[off] = static_cast<float>(y_gossip);
+            continue;
+          }
+          if (p.mode == kModeDpsgd) {
+            const double x_new = cx[i * S + col] - alpha * static_cast<double>(p.g[off]);
+            const float x_new_f = static_cast<float>(x_new);
+            const double g_new = fma(static_cast<double>(p.a[off]), x_new - static_cast<double>(p.c[off]),
+                                     sigma * static_cast<double>(xi[w]));
+            p.x[off] = x_new_f;
+            p.g[off] = static_cast<float>(g_new);
+            continue;
+          }
           const double y_gossip = cy[i * S + col];
           const double x_new = cx[i * S + col] - alpha * y_gossip;
           // gradient point: the new model, or (Algorithm 2 as printed) the model this step started from,
@@ -145,11 +168,10 @@ int plan_step_csr(StepParams& p, int smem_optin_bytes) {
 
 int launch_step_csr(const StepParams& p, int sm_count, cudaStream_t stream) {
   const size_t smem = csr_smem_bytes(p.n, p.nnz, p.S);
-  cudaError_t e = cudaFuncSetAttribute(step_csr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem));
-  if (e != cudaSuccess) return static_cast<int>(e);
+  const int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(step_csr_kernel), static_cast<int>(smem));
+  if (rc != 0) return rc;
   int per_sm = 1;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, step_csr_kernel, kCsrThreads, smem);
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, step_csr_kernel, kCsrThreads, smem);
   if (e != cudaSuccess) return static_cast<int>(e);
   if (per_sm < 1) per_sm = 1;
   const long long grid = p.num_slabs < static_cast<long long>(sm_count) * per_sm

@@ -31,114 +31,39 @@
 //             TMA tile stores.  Row-contiguous 256-byte writes matter: storing straight from the
 //             accumulator layout (32-byte pieces of 8 rows per instruction) halves the HBM throughput.
 // Every mbarrier wait is bounded; a wait that gives up sets the status word and the CTA winds down.
+//
+// Modes (template parameter): the DeTAG step with the library's synthetic gradient (above); the DeTAG step with
+// caller-written gradients (Algorithm 2's tracker update y + g_new - g_old forms the B operand of the tracker
+// contraction, the tail only rounds and copies g_new over g_old); and D-PSGD (one contraction: x' = P x - alpha g,
+// no tracker).
 #include "mma_common.cuh"
 
 namespace detag {
 
 namespace {
 
+// kMode: what the step computes (kModeDetag / kModeExternal / kModeDpsgd).
 // kAtStart: the gradient is taken at the model the step started from (Algorithm 2 as printed) instead of the new one.
 // kKs: number of 4-worker input blocks that can be non-zero, ceil(n / 4) rounded up to 2, 4 or 8; the MMAs of the
 // all-zero blocks of the padded P are not issued.
-template <bool kAtStart, int kKs>
+template <int kMode, bool kAtStart, int kKs>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
   // No static shared memory in this kernel: the dynamic array starts at the CTA's shared window, whose
-  // 128-byte alignment (needed by the TMA tiles) is checked below rather than assumed.
+  // 128-byte alignment (needed by the TMA tiles) is checked in the set-up rather than assumed.
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  float* stage_mem = reinterpret_cast<float*>(smem_raw);
-  float* out_mem = stage_mem + kMmaStages * kStageFloats;                             // [group][x', y', g'][32][kS]
-  double* frag = reinterpret_cast<double*>(out_mem + kWarpGroups * kOutFloats);       // [t][ks][lane]
-  uint64_t* full = reinterpret_cast<uint64_t*>(frag + 32 * 32);
-  uint64_t* empty = full + kMmaStages;
-  uint64_t* out_ready = empty + kMmaStages;      // [group]: the group's 8 warps have written their outputs
-  uint64_t* out_free = out_ready + kWarpGroups;  // [group]: the stores have finished reading the tile
-  unsigned* seen = reinterpret_cast<unsigned*>(out_free + kWarpGroups);  // [group]: 1 + last slab index whose data it saw
-  if ((s_addr(smem_raw) & 127u) != 0) {
-    if (threadIdx.x == 0) atomicExch(p.status, 2);
-    return;
-  }
-
+  MmaShared sm;
+  if (!mma_setup(p, smem_raw, sm)) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = p.n;
-  // P in fragment order: block (t, ks), lane (r, kq) holds P[4r + t][4ks + kq]
-  for (int e = tid; e < 32 * 32; e += kMmaThreads) {
-    const int l = e & 31, ks = (e >> 5) & 7, t = e >> 8;
-    const int i = 4 * (l >> 2) + t, j = 4 * ks + (l & 3);
-    frag[e] = (i < n && j < n) ? p.poly[static_cast<size_t>(i) * n + j] : 0.0;
-  }
-  if (tid == 0) {
-    for (int g = 0; g < kWarpGroups; ++g) seen[g] = 0;
-    for (int s = 0; s < kMmaStages; ++s) {
-      bar_init(&full[s], 1);
-      bar_init(&empty[s], kGroupWarps);
-    }
-    for (int g = 0; g < kWarpGroups; ++g) {
-      bar_init(&out_ready[g], kGroupWarps);
-      bar_init(&out_free[g], 1);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  __syncthreads();
-
   const long long first = blockIdx.x, stride = gridDim.x;
 
   if (warp == kProducerWarp) {
-    // ---------------------------------------------------------------- producer: one elected thread
-    if (lane == 0) {
-      int issued = 0;
-      bool ok = true;
-      for (long long slab = first; slab < p.num_slabs; slab += stride, ++issued) {
-        const int s = issued % kMmaStages;
-        if (issued >= kMmaStages) ok = bar_wait(&empty[s], ((issued / kMmaStages) - 1) & 1);
-        if (!ok) break;
-        float* st = stage_mem + static_cast<size_t>(s) * kStageFloats;
-        const int col = static_cast<int>(slab * kS);
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_addr(&full[s])),
-                     "r"(static_cast<unsigned>(kStageBytes))
-                     : "memory");
-        tile_load(st, &maps.x, col, &full[s]);
-        tile_load(st + kN * kPitchXY, &maps.y, col, &full[s]);
-        float* se = st + 2 * kN * kPitchXY;
-        tile_load(se, &maps.g, col, &full[s]);
-        tile_load(se + kN * kPitchE, &maps.a, col, &full[s]);
-        tile_load(se + 2 * kN * kPitchE, &maps.c, col, &full[s]);
-      }
-      if (!ok) {
-        atomicExch(p.status, 1);
-        for (int back = 1; back <= kMmaStages && back <= issued; ++back) {  // drain copies still in flight (bounded)
-          const int k = issued - back;
-          bar_wait(&full[k % kMmaStages], (k / kMmaStages) & 1);
-        }
-      }
-    }
+    if (lane == 0) mma_producer<kMode>(p, maps, sm);
     return;
   }
-
   if (warp == kStoreWarp) {
-    // ---------------------------------------------------------------- storer: one elected thread
-    if (lane == 0) {
-      long long k = 0;
-      for (long long slab = first; slab < p.num_slabs; slab += stride, ++k) {
-        const int g = static_cast<int>(k % kWarpGroups);
-        if (!bar_wait(&out_ready[g], (k / kWarpGroups) & 1)) {
-          atomicExch(p.status, 1);
-          break;
-        }
-        const float* ob = out_mem + g * kOutFloats;
-        const int col = static_cast<int>(slab * kS);
-        if (col < (p.d & ~3LL)) {
-          tile_store(&maps.xs, col, ob);
-          tile_store(&maps.ys, col, ob + kN * kS);
-          tile_store(&maps.gs, col, ob + 2 * kN * kS);
-        }
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // the tile may be overwritten now
-        bar_arrive(&out_free[g]);
-      }
-      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // all global writes done before the CTA leaves
-    }
+    if (lane == 0) mma_storer<kMode>(p, maps, sm);
     return;
   }
 
@@ -148,7 +73,7 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
   const double alpha = p.alpha;
   const float sigma = static_cast<float>(p.sigma);
   const bool noisy = p.sigma != 0.0;
-  float* ob = out_mem + group * kOutFloats;
+  float* ob = sm.out_mem + group * kOutFloats;
   const int cl = tile * 8;
   const long long d_tma = p.d & ~3LL;  // columns below this are written by the TMA stores
 
@@ -156,25 +81,14 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
   for (long long k = group, slab = first + group * stride; slab < p.num_slabs;
        slab += kWarpGroups * stride, k += kWarpGroups, ++use) {
     const int s = static_cast<int>(k % kMmaStages);
-    bool ok = true;
-    if (lane == 0) {
-      // The stage last held slab k - kMmaStages, which belongs to the other group when the stage count is odd.
-      // A parity wait must not start before that phase has completed (it could not tell the two apart), and
-      // it costs nothing to make sure: this slab cannot have been loaded before that one was consumed.
-      if (kMmaStages % kWarpGroups != 0 && k >= kMmaStages)
-        ok = count_wait(&seen[(k - kMmaStages) % kWarpGroups], static_cast<unsigned>(k - kMmaStages + 1));
-      if (ok) ok = bar_wait(&full[s], (k / kMmaStages) & 1);
-      if (ok && tile == 0) count_publish(&seen[group], static_cast<unsigned>(k + 1));
-    }
-    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-    if (!ok) {
+    if (!mma_wait_slab(p, sm, k, group, tile, lane)) {
       if (lane == 0) atomicExch(p.status, 1);
       return;
     }
-    const float* sx = stage_mem + static_cast<size_t>(s) * kStageFloats;
+    const float* sx = sm.stage_mem + static_cast<size_t>(s) * kStageFloats;
     const float* sy = sx + kN * kPitchXY;
     const float* sg = sy + kN * kPitchXY;
-    const float* sa = sg + kN * kPitchE;
+    const float* sa = sg + kN * kPitchE;  // objective data a, or the caller's newest gradient
     const float* sc = sa + kN * kPitchE;
     const long long j0 = slab * kS;
 
@@ -186,23 +100,42 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
       //   cy starts at -g and accumulates P y, ending as y~ - g    (so the fold is y' = cy + g')
       // Scalar float64 operations share the FP64 tensor pipe with the MMAs; every one issued from the tail
       // queues behind other warps' MMAs, so as many as possible are done here, where this warp holds the pipe.
+      // Caller-written gradients: the tracker operand is folded here, y + (g_new - g_old), and cy starts at 0.
+      // D-PSGD: cx starts at -alpha g and accumulates P x; there is no tracker.
       double cy[4][2], cx[4][2];
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
-        const float2 gv = *reinterpret_cast<const float2*>(sg + (4 * r + t) * kPitchE + cl + 2 * kq);
-        cy[t][0] = static_cast<double>(-gv.x);
-        cy[t][1] = static_cast<double>(-gv.y);
+        cy[t][0] = cy[t][1] = 0.0;
         cx[t][0] = cx[t][1] = 0.0;
+        if (kMode != kModeExternal) {
+          const float2 gv = *reinterpret_cast<const float2*>(sg + (4 * r + t) * kPitchE + cl + 2 * kq);
+          if (kMode == kModeDetag) {
+            cy[t][0] = static_cast<double>(-gv.x);
+            cy[t][1] = static_cast<double>(-gv.y);
+          } else {
+            cx[t][0] = -alpha * static_cast<double>(gv.x);
+            cx[t][1] = -alpha * static_cast<double>(gv.y);
+          }
+        }
       }
 #pragma unroll
       for (int ks = 0; ks < kKs; ++ks) {
         const int src = (4 * ks + kq) * kPitchXY + cl + r;
-        const double by = static_cast<double>(sy[src]);
-        const double bx = fma(-alpha, by, static_cast<double>(sx[src]));
+        double by = 0.0, bx;
+        if (kMode == kModeDpsgd) {
+          bx = static_cast<double>(sx[src]);
+        } else {
+          by = static_cast<double>(sy[src]);
+          if (kMode == kModeExternal) {
+            const int esrc = (4 * ks + kq) * kPitchE + cl + r;
+            by += static_cast<double>(sa[esrc]) - static_cast<double>(sg[esrc]);  // Algorithm 2's tracker update
+          }
+          bx = fma(-alpha, by, static_cast<double>(sx[src]));
+        }
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-          const double a = frag[(t * 8 + ks) * 32 + lane];
-          dmma(cy[t], a, by);
+          const double a = sm.frag[(t * 8 + ks) * 32 + lane];
+          if (kMode != kModeDpsgd) dmma(cy[t], a, by);
           dmma(cx[t], a, bx);
         }
       }
@@ -212,14 +145,14 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
       for (int t = 0; t < 4; ++t) {
         const int eoff = (4 * r + t) * kPitchE + cl + 2 * kq;
         av4[t] = *reinterpret_cast<const float2*>(sa + eoff);
-        cv4[t] = *reinterpret_cast<const float2*>(sc + eoff);
-        if (p.y_obs != nullptr) gv4[t] = *reinterpret_cast<const float2*>(sg + eoff);
+        if (kMode != kModeExternal) cv4[t] = *reinterpret_cast<const float2*>(sc + eoff);
+        if (kMode == kModeDetag && p.y_obs != nullptr) gv4[t] = *reinterpret_cast<const float2*>(sg + eoff);
       }
       __syncwarp();
       if (lane == 0) {
-        bar_arrive(&empty[s]);
+        bar_arrive(&sm.empty[s]);
         released = true;
-        if (use > 0 && !bar_wait(&out_free[group], (use - 1) & 1)) out_ok = false;  // previous tile stored
+        if (use > 0 && !bar_wait(&sm.out_free[group], (use - 1) & 1, p.spin_limit)) out_ok = false;  // previous tile stored
       }
       out_ok = __shfl_sync(0xffffffffu, out_ok ? 1 : 0, 0) != 0;
       if (!out_ok) {
@@ -231,7 +164,7 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
       float xi[2][4];
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        if (noisy) {
+        if (kMode != kModeExternal && noisy) {
           normal_quad(p.seed_lo, p.seed_hi, static_cast<unsigned long long>(p.coord_offset + j + e),
                       static_cast<uint32_t>(r), p.t_noise, xi[e]);
         } else {
@@ -241,26 +174,31 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const int row = 4 * r + t;
-        const int eoff = row * kPitchE + cl + 2 * kq;
         const float2 av = av4[t];
-        const float2 cv = cv4[t];
         float2 xo, yo, go;
         xo.x = static_cast<float>(cx[t][0]);                           // x' (float64 accumulator, rounded once)
         xo.y = static_cast<float>(cx[t][1]);
-        float2 x_at = xo;  // gradient point: the new model, or (Algorithm 2 as printed) the model before this step.
-        if (kAtStart && row < n) {
-          // The old model is still in global memory: this slab's stores are issued after all of its tails.
-          const long long off = static_cast<long long>(row) * p.ld + j;
-          x_at.x = j < p.d ? p.x[off] : 0.f;
-          x_at.y = j + 1 < p.d ? p.x[off + 1] : 0.f;
+        if (kMode == kModeExternal) {
+          go = av;                                                     // the gradient just folded becomes g_old
+          yo.x = static_cast<float>(cy[t][0]);                         // the gossiped tracker
+          yo.y = static_cast<float>(cy[t][1]);
+        } else {
+          const float2 cv = cv4[t];
+          float2 x_at = xo;  // gradient point: the new model, or (Algorithm 2 as printed) the model before this step.
+          if (kAtStart && row < n) {
+            // The old model is still in global memory: this slab's stores are issued after all of its tails.
+            const long long off = static_cast<long long>(row) * p.ld + j;
+            x_at.x = j < p.d ? p.x[off] : 0.f;
+            x_at.y = j + 1 < p.d ? p.x[off + 1] : 0.f;
+          }
+          go.x = fmaf(av.x, x_at.x - cv.x, sigma * xi[0][t]);            // stochastic gradient
+          go.y = fmaf(av.y, x_at.y - cv.y, sigma * xi[1][t]);
+          yo.x = static_cast<float>(cy[t][0] + static_cast<double>(go.x));  // fold: (y~ - g) + g', g' as stored
+          yo.y = static_cast<float>(cy[t][1] + static_cast<double>(go.y));
         }
-        go.x = fmaf(av.x, x_at.x - cv.x, sigma * xi[0][t]);            // stochastic gradient
-        go.y = fmaf(av.y, x_at.y - cv.y, sigma * xi[1][t]);
-        yo.x = static_cast<float>(cy[t][0] + static_cast<double>(go.x));  // fold: (y~ - g) + g', g' as stored
-        yo.y = static_cast<float>(cy[t][1] + static_cast<double>(go.y));
         const int ooff = row * kS + cl + 2 * kq;
         *reinterpret_cast<float2*>(ob + ooff) = xo;
-        *reinterpret_cast<float2*>(ob + kN * kS + ooff) = yo;
+        if (kMode != kModeDpsgd) *reinterpret_cast<float2*>(ob + kN * kS + ooff) = yo;
         *reinterpret_cast<float2*>(ob + 2 * kN * kS + ooff) = go;
         if (j >= d_tma && row < n) {
           // TMA clips a store at 16-byte granularity; the last d % 4 coordinates are written here so that
@@ -268,61 +206,82 @@ step_mma_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
           const long long off = static_cast<long long>(row) * p.ld + j;
           if (j < p.d) {
             p.x[off] = xo.x;
-            p.y[off] = yo.x;
+            if (kMode != kModeDpsgd) p.y[off] = yo.x;
             p.g[off] = go.x;
           }
           if (j + 1 < p.d) {
             p.x[off + 1] = xo.y;
-            p.y[off + 1] = yo.y;
+            if (kMode != kModeDpsgd) p.y[off + 1] = yo.y;
             p.g[off + 1] = go.y;
           }
         }
-        if (p.y_obs != nullptr && row < n) {  // optional observer: the gossiped tracker, stored directly
+        if (kMode != kModeDpsgd && p.y_obs != nullptr && row < n) {  // optional observer: the gossiped tracker, stored directly
           const long long off = static_cast<long long>(row) * p.ld + j;
-          const float2 gv = gv4[t];
+          float2 yg = yo;
+          if (kMode == kModeDetag) {
+            const float2 gv = gv4[t];
+            yg = make_float2(static_cast<float>(cy[t][0] + static_cast<double>(gv.x)),
+                             static_cast<float>(cy[t][1] + static_cast<double>(gv.y)));
+          }
           if (j + 1 < p.d) {
-            *reinterpret_cast<float2*>(p.y_obs + off) =
-                make_float2(static_cast<float>(cy[t][0] + static_cast<double>(gv.x)),
-                            static_cast<float>(cy[t][1] + static_cast<double>(gv.y)));
+            *reinterpret_cast<float2*>(p.y_obs + off) = yg;
           } else if (j < p.d) {
-            p.y_obs[off] = static_cast<float>(cy[t][0] + static_cast<double>(gv.x));
+            p.y_obs[off] = yg.x;
           }
         }
       }
     }
     // outputs visible to the TMA store
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    fence_async_shared();
     __syncwarp();
     if (!(j0 + cl < p.d)) {  // idle tile
-      if (lane == 0 && use > 0 && !bar_wait(&out_free[group], (use - 1) & 1)) atomicExch(p.status, 1);
+      if (lane == 0 && use > 0 && !bar_wait(&sm.out_free[group], (use - 1) & 1, p.spin_limit)) atomicExch(p.status, 1);
     }
     if (lane == 0) {
-      bar_arrive(&out_ready[group]);
-      if (!released) bar_arrive(&empty[s]);
+      bar_arrive(&sm.out_ready[group]);
+      if (!released) bar_arrive(&sm.empty[s]);
     }
   }
 }
 
+typedef void (*MmaKernel)(const StepParams, const MmaMaps);
+
+template <int kKs>
+MmaKernel pick_mode(const StepParams& p) {
+  if (p.mode == kModeExternal) return step_mma_kernel<kModeExternal, false, kKs>;
+  if (p.mode == kModeDpsgd) return step_mma_kernel<kModeDpsgd, false, kKs>;
+  return p.grad_at_start ? step_mma_kernel<kModeDetag, true, kKs> : step_mma_kernel<kModeDetag, false, kKs>;
+}
+
 }  // namespace
 
-int launch_step_mma(StepParams p, int sm_count, cudaStream_t stream) {
-  MmaMaps maps;
-  if (!make_mma_maps(&maps, p)) return static_cast<int>(cudaErrorInvalidValue);
+// Tensor maps over the arrays in `p`; false when the driver refuses one.
+bool build_maps_mma(const StepParams& p, TensorMapSet* out) {
+  MmaMaps* maps = reinterpret_cast<MmaMaps*>(out->bytes);
+  const float* slot_a = p.mode == kModeExternal ? p.g_ext : p.a;
+  const float* slot_c = p.mode == kModeExternal ? p.g_ext : p.c;
+  const float* y = p.mode == kModeDpsgd ? p.x : p.y;  // D-PSGD has no tracker: the map is never used
+  if (!make_map(&maps->x, p.x, p.n, p.d, p.ld, kN, kPitchXY) || !make_map(&maps->y, y, p.n, p.d, p.ld, kN, kPitchXY) ||
+      !make_map(&maps->g, p.g, p.n, p.d, p.ld, kN, kPitchE) || !make_map(&maps->a, slot_a, p.n, p.d, p.ld, kN, kPitchE) ||
+      !make_map(&maps->c, slot_c, p.n, p.d, p.ld, kN, kPitchE))
+    return false;
+  const long long d_tma = p.d & ~3LL;  // the stores' tensor ends on a 16-byte boundary (see the kernels' tails)
+  if (d_tma > 0 && (!make_map(&maps->xs, p.x, p.n, d_tma, p.ld, kN, kS) || !make_map(&maps->ys, y, p.n, d_tma, p.ld, kN, kS) ||
+                    !make_map(&maps->gs, p.g, p.n, d_tma, p.ld, kN, kS)))
+    return false;
+  if (d_tma == 0) maps->xs = maps->ys = maps->gs = maps->x;  // never used: every slab lies beyond column 0
+  return true;
+}
+
+int launch_step_mma(StepParams p, const TensorMapSet& maps, int sm_count, cudaStream_t stream) {
   p.S = kS;
   p.num_slabs = (p.d + kS - 1) / kS;
-  void (*kernel)(const StepParams, const MmaMaps);
-  if (p.n <= 8)
-    kernel = p.grad_at_start ? step_mma_kernel<true, 2> : step_mma_kernel<false, 2>;
-  else if (p.n <= 16)
-    kernel = p.grad_at_start ? step_mma_kernel<true, 4> : step_mma_kernel<false, 4>;
-  else
-    kernel = p.grad_at_start ? step_mma_kernel<true, 8> : step_mma_kernel<false, 8>;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(kMmaSmemBytes));
-  if (e != cudaSuccess) return static_cast<int>(e);
+  const MmaKernel kernel = p.n <= 8 ? pick_mode<2>(p) : p.n <= 16 ? pick_mode<4>(p) : pick_mode<8>(p);
+  const int e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), static_cast<int>(kMmaSmemBytes));
+  if (e != 0) return e;
   const long long grid = p.num_slabs < sm_count ? p.num_slabs : sm_count;
   if (grid <= 0) return 0;
-  kernel<<<static_cast<unsigned>(grid), kMmaThreads, kMmaSmemBytes, stream>>>(p, maps);
+  kernel<<<static_cast<unsigned>(grid), kMmaThreads, kMmaSmemBytes, stream>>>(p, *reinterpret_cast<const MmaMaps*>(maps.bytes));
   return static_cast<int>(cudaGetLastError());
 }
 

@@ -24,101 +24,25 @@ template <bool kAtStart, int kKs>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 step_mma_many_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
   // No static shared memory in this kernel: the dynamic array starts at the CTA's shared window, whose
-  // 128-byte alignment (needed by the TMA tiles) is checked below rather than assumed.
+  // 128-byte alignment (needed by the TMA tiles) is checked in the set-up rather than assumed.
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  float* stage_mem = reinterpret_cast<float*>(smem_raw);
-  float* out_mem = stage_mem + kMmaStages * kStageFloats;                             // [group][x', y', g'][32][kS]
-  double* frag = reinterpret_cast<double*>(out_mem + kWarpGroups * kOutFloats);       // [t][ks][lane]
-  uint64_t* full = reinterpret_cast<uint64_t*>(frag + 32 * 32);
-  uint64_t* empty = full + kMmaStages;
-  uint64_t* out_ready = empty + kMmaStages;      // [group]: the group's 8 warps have written their outputs
-  uint64_t* out_free = out_ready + kWarpGroups;  // [group]: the stores have finished reading the tile
-  unsigned* seen = reinterpret_cast<unsigned*>(out_free + kWarpGroups);  // [group]: 1 + last slab index whose data it saw
-  if ((s_addr(smem_raw) & 127u) != 0) {
-    if (threadIdx.x == 0) atomicExch(p.status, 2);
-    return;
-  }
-
+  MmaShared sm;
+  if (!mma_setup(p, smem_raw, sm)) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = p.n;
-  // P in fragment order: block (t, ks), lane (r, kq) holds P[4r + t][4ks + kq]
-  for (int e = tid; e < 32 * 32; e += kMmaThreads) {
-    const int l = e & 31, ks = (e >> 5) & 7, t = e >> 8;
-    const int i = 4 * (l >> 2) + t, j = 4 * ks + (l & 3);
-    frag[e] = (i < n && j < n) ? p.poly[static_cast<size_t>(i) * n + j] : 0.0;
-  }
-  if (tid == 0) {
-    for (int g = 0; g < kWarpGroups; ++g) seen[g] = 0;
-    for (int s = 0; s < kMmaStages; ++s) {
-      bar_init(&full[s], 1);
-      bar_init(&empty[s], kGroupWarps);
-    }
-    for (int g = 0; g < kWarpGroups; ++g) {
-      bar_init(&out_ready[g], kGroupWarps);
-      bar_init(&out_free[g], 1);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  __syncthreads();
-
   const long long first = blockIdx.x, stride = gridDim.x;
+  float* const stage_mem = sm.stage_mem;
+  uint64_t* const empty = sm.empty;
+  uint64_t* const out_ready = sm.out_ready;
+  uint64_t* const out_free = sm.out_free;
+  const double* const frag = sm.frag;
 
   if (warp == kProducerWarp) {
-    // ---------------------------------------------------------------- producer: one elected thread
-    if (lane == 0) {
-      int issued = 0;
-      bool ok = true;
-      for (long long slab = first; slab < p.num_slabs; slab += stride, ++issued) {
-        const int s = issued % kMmaStages;
-        if (issued >= kMmaStages) ok = bar_wait(&empty[s], ((issued / kMmaStages) - 1) & 1);
-        if (!ok) break;
-        float* st = stage_mem + static_cast<size_t>(s) * kStageFloats;
-        const int col = static_cast<int>(slab * kS);
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_addr(&full[s])),
-                     "r"(static_cast<unsigned>(kStageBytes))
-                     : "memory");
-        tile_load(st, &maps.x, col, &full[s]);
-        tile_load(st + kN * kPitchXY, &maps.y, col, &full[s]);
-        float* se = st + 2 * kN * kPitchXY;
-        tile_load(se, &maps.g, col, &full[s]);
-        tile_load(se + kN * kPitchE, &maps.a, col, &full[s]);
-        tile_load(se + 2 * kN * kPitchE, &maps.c, col, &full[s]);
-      }
-      if (!ok) {
-        atomicExch(p.status, 1);
-        for (int back = 1; back <= kMmaStages && back <= issued; ++back) {  // drain copies still in flight (bounded)
-          const int k = issued - back;
-          bar_wait(&full[k % kMmaStages], (k / kMmaStages) & 1);
-        }
-      }
-    }
+    if (lane == 0) mma_producer<kModeDetag>(p, maps, sm);
     return;
   }
-
   if (warp == kStoreWarp) {
-    // ---------------------------------------------------------------- storer: one elected thread
-    if (lane == 0) {
-      long long k = 0;
-      for (long long slab = first; slab < p.num_slabs; slab += stride, ++k) {
-        const int g = static_cast<int>(k % kWarpGroups);
-        if (!bar_wait(&out_ready[g], (k / kWarpGroups) & 1)) {
-          atomicExch(p.status, 1);
-          break;
-        }
-        const float* ob = out_mem + g * kOutFloats;
-        const int col = static_cast<int>(slab * kS);
-        if (col < (p.d & ~3LL)) {
-          tile_store(&maps.xs, col, ob);
-          tile_store(&maps.ys, col, ob + kN * kS);
-          tile_store(&maps.gs, col, ob + 2 * kN * kS);
-        }
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // the tile may be overwritten now
-        bar_arrive(&out_free[g]);
-      }
-      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // all global writes done before the CTA leaves
-    }
+    if (lane == 0) mma_storer<kModeDetag>(p, maps, sm);
     return;
   }
 
@@ -128,7 +52,7 @@ step_mma_many_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
   const double alpha = p.alpha;
   const float sigma = static_cast<float>(p.sigma);
   const bool noisy = p.sigma != 0.0;
-  float* ob = out_mem + group * kOutFloats;
+  float* ob = sm.out_mem + group * kOutFloats;
   const int cl = tile * 8;
   const long long d_tma = p.d & ~3LL;  // columns below this are written by the TMA stores
   const int steps = p.steps;
@@ -138,15 +62,7 @@ step_mma_many_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
        slab += kWarpGroups * stride, k += kWarpGroups, ++use) {
     const int s = static_cast<int>(k % kMmaStages);
     bool ok = true;
-    if (lane == 0) {
-      // see step_mma.cu: a parity wait on a stage shared with the other group must not start a phase early
-      if (kMmaStages % kWarpGroups != 0 && k >= kMmaStages)
-        ok = count_wait(&seen[(k - kMmaStages) % kWarpGroups], static_cast<unsigned>(k - kMmaStages + 1));
-      if (ok) ok = bar_wait(&full[s], (k / kMmaStages) & 1);
-      if (ok && tile == 0) count_publish(&seen[group], static_cast<unsigned>(k + 1));
-    }
-    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-    if (!ok) {
+    if (!mma_wait_slab(p, sm, k, group, tile, lane)) {
       if (lane == 0) atomicExch(p.status, 1);
       return;
     }
@@ -183,7 +99,7 @@ step_mma_many_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
           }
         }
         if (final_step && use > 0) {  // the group's output tile must have been read by the previous stores
-          if (lane == 0) ok = bar_wait(&out_free[group], (use - 1) & 1);
+          if (lane == 0) ok = bar_wait(&out_free[group], (use - 1) & 1, p.spin_limit);
           ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
           if (!ok) {
             if (lane == 0) atomicExch(p.status, 1);
@@ -247,10 +163,10 @@ step_mma_many_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
         __syncwarp();  // the new state is in place before the next step's fragment loads
       }
     } else if (use > 0) {  // idle tile: same protocol, nothing computed
-      if (lane == 0 && !bar_wait(&out_free[group], (use - 1) & 1)) atomicExch(p.status, 1);
+      if (lane == 0 && !bar_wait(&out_free[group], (use - 1) & 1, p.spin_limit)) atomicExch(p.status, 1);
     }
     // outputs visible to the TMA store, input stage no longer read or written by this warp
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    fence_async_shared();
     __syncwarp();
     if (lane == 0) {
       bar_arrive(&out_ready[group]);
@@ -261,9 +177,8 @@ step_mma_many_kernel(const StepParams p, const __grid_constant__ MmaMaps maps) {
 
 }  // namespace
 
-int launch_step_mma_many(StepParams p, int sm_count, cudaStream_t stream) {
-  MmaMaps maps;
-  if (p.steps < 1 || !make_mma_maps(&maps, p)) return static_cast<int>(cudaErrorInvalidValue);
+int launch_step_mma_many(StepParams p, const TensorMapSet& maps, int sm_count, cudaStream_t stream) {
+  if (p.steps < 1 || p.mode != kModeDetag) return static_cast<int>(cudaErrorInvalidValue);
   p.S = kS;
   p.num_slabs = (p.d + kS - 1) / kS;
   void (*kernel)(const StepParams, const MmaMaps);
@@ -273,12 +188,11 @@ int launch_step_mma_many(StepParams p, int sm_count, cudaStream_t stream) {
     kernel = p.grad_at_start ? step_mma_many_kernel<true, 4> : step_mma_many_kernel<false, 4>;
   else
     kernel = p.grad_at_start ? step_mma_many_kernel<true, 8> : step_mma_many_kernel<false, 8>;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(kMmaSmemBytes));
-  if (e != cudaSuccess) return static_cast<int>(e);
+  const int e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), static_cast<int>(kMmaSmemBytes));
+  if (e != 0) return e;
   const long long grid = p.num_slabs < sm_count ? p.num_slabs : sm_count;
   if (grid <= 0) return 0;
-  kernel<<<static_cast<unsigned>(grid), kMmaThreads, kMmaSmemBytes, stream>>>(p, maps);
+  kernel<<<static_cast<unsigned>(grid), kMmaThreads, kMmaSmemBytes, stream>>>(p, *reinterpret_cast<const MmaMaps*>(maps.bytes));
   return static_cast<int>(cudaGetLastError());
 }
 

@@ -18,13 +18,15 @@ class Session:
 
     ``m`` is the matrix a gossip round applies row-wise (an ``inputs.CSR``); ``a``, ``c``, ``x0`` are
     host float32 arrays of shape [n, d] (or None to leave the device buffers uninitialised, e.g.
-    when they are filled on the device).
+    when they are filled on the device).  ``external_gradient`` adds the buffer ``g_new`` for
+    caller-written gradients and selects that source.
     """
 
     def __init__(self, m, d: int, K: int, eta: float, alpha: float, a=None, c=None, x0=None, sigma: float = 0.0,
                  seed: int = 0, coord_offset: int = 0, ld: Optional[int] = None, device: str = "cuda:0",
                  observe_gossip: bool = False, variant: int = B.DETAG_VARIANT_AUTO,
-                 gradient_point: int = B.DETAG_GRADIENT_AT_NEW_MODEL):
+                 gradient_point: int = B.DETAG_GRADIENT_AT_NEW_MODEL, algorithm: int = B.DETAG_ALGORITHM_DETAG,
+                 external_gradient: bool = False):
         import torch
 
         if not torch.cuda.is_available():
@@ -57,6 +59,12 @@ class Session:
             B.detag_set_variant(self.state, variant)
         if gradient_point != B.DETAG_GRADIENT_AT_NEW_MODEL:
             B.detag_set_gradient_point(self.state, gradient_point)
+        if algorithm != B.DETAG_ALGORITHM_DETAG:
+            B.detag_set_algorithm(self.state, algorithm)
+        # caller-written gradients: the array the caller fills before init and before every step
+        self.g_new = torch.zeros(shape, dtype=torch.float32, device=self.device) if external_gradient else None
+        if external_gradient:
+            B.detag_set_gradient_source(self.state, B.DETAG_GRADIENT_EXTERNAL, self.g_new)
 
     # ---- data movement (plumbing only)
     def upload(self, name: str, host) -> None:

@@ -132,12 +132,41 @@ def test_average_consensus_and_dsgt_special_cases():
     _check_one_step(inputs.metropolis_weights(inputs.ring_graph(6)), 1, 0.0, 0.1, a, c, x0, 0.1, 1)  # DSGT
 
 
-def test_coordinate_offset_enters_the_noise_counter():
-    rng = np.random.default_rng(8)
-    m = inputs.metropolis_weights(inputs.ring_graph(8))
-    a, c = _random_objective(rng, 8, 64)
-    x0 = np.zeros((8, 64), dtype=np.float32)
-    _check_one_step(m, 2, 0.25, 0.05, a, c, x0, 0.1, 9, j0=(1 << 32) + 12345, variants=[B.DETAG_VARIANT_CSR])
+@pytest.mark.parametrize("n,d,K", [(8, 64, 2), (16, 130, 3), (32, 257, 2), (40, 70, 2), (64, 130, 4), (96, 67, 3)])
+def test_coordinate_offset_enters_the_noise_counter(n, d, K):
+    """Column offsets beyond 2^32 reach the high word of the noise counter in every kernel variant that accepts
+    the matrix (each kernel forms coord_offset + j on its own)."""
+    rng = np.random.default_rng(8 + n)
+    m = inputs.metropolis_weights(inputs.ring_graph(n))
+    a, c = _random_objective(rng, n, d, scale=0.2)
+    x0 = np.zeros((n, d), dtype=np.float32)
+    for j0 in ((1 << 32) + 12345, (5 << 32) - 17):  # the second one crosses a multiple of 2^32 inside the arrays
+        _check_one_step(m, K, 0.25, 0.05, a, c, x0, 0.1, 9, j0=j0)
+
+
+def test_coordinate_offset_in_the_fused_multi_step_call():
+    """detag_step_many forms its own noise counters: with an offset beyond 2^32 it must still equal the oracle."""
+    rng = np.random.default_rng(21)
+    n, d, K, j0 = 16, 1000, 3, (3 << 32) + 999
+    m = inputs.metropolis_weights(inputs.ring_graph(n))
+    eta = orc.spectrum(m.to_dense()).eta
+    a, c = _random_objective(rng, n, d)
+    x0 = rng.standard_normal((n, d)).astype(np.float32)
+    p = oracle_problem(m, K, eta, 0.05, a, c, 0.1, 4, j0)
+    ref = orc.run(p, x0, 6)
+    with Session(m, d, K, eta, 0.05, a, c, x0, 0.1, 4, coord_offset=j0) as s:
+        assert B.detag_get_variant(s.state) == B.DETAG_VARIANT_DENSE
+        s.init()
+        s.step_many(6)
+        s.status()
+        for k, want in (("x", ref.x), ("y", orc.folded_tracker(ref)), ("g", ref.g_new)):
+            assert rel_l2(s.download(k), want) <= 1e-4, k
+        # noise is what distinguishes offsets: the same run at offset 0 must differ
+        got_g = s.download("g")
+    with Session(m, d, K, eta, 0.05, a, c, x0, 0.1, 4, coord_offset=j0 - (3 << 32)) as s:
+        s.init()
+        s.step_many(6)
+        assert not np.array_equal(s.download("g"), got_g)
 
 
 def test_padded_leading_dimension_is_left_untouched():

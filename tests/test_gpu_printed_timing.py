@@ -85,7 +85,7 @@ def test_small_rings_ragged_sizes(n, d, K):
     _check_trajectory(m, K, eta, 0.05, a, c, x0, 0.1, 13, 6, variants)
 
 
-def test_torus_64_register_tiled_kernel():
+def test_torus_64_dense_polynomial_kernel():
     rng = np.random.default_rng(64)
     m = inputs.gossip_matrix(inputs.CONFIGS["cfg3"])
     eta = orc.spectrum(m.to_dense()).eta

@@ -432,6 +432,70 @@ def test_printed_timing_differs_from_the_fresh_gradient_step_only_by_the_gradien
     assert np.allclose(nxt.y, orc.fold(y_gossip, orc.gradient(s.x, p.a, p.c, 0.0, None), s.g_prev), atol=1e-13)
 
 
+# ----------------------------------------------------------------------------- D-PSGD
+def test_dpsgd_matches_the_affine_recursion_in_dense_matrix_powers():
+    """Noise free, one coordinate at a time the iteration is affine: x' = (P - alpha D_a) x + alpha D_a c with
+    P from brute-force matrix products, so x_T = B^T x_0 + (sum_{k<T} B^k) alpha D_a c by explicit powers."""
+    p, w = _small_problem(21, n=7, m=5, K=2, sigma=0.0, alpha=0.04)
+    P = _dense_polynomial(w.to_dense(), p.K, p.eta)
+    x0 = np.random.default_rng(2).standard_normal((7, 5))
+    T = 6
+    s = orc.run_dpsgd(p, x0, T)
+    a, c = p.a.astype(np.float64), p.c.astype(np.float64)
+    for j in range(5):
+        B = P - p.alpha * np.diag(a[:, j])
+        acc = sum(np.linalg.matrix_power(B, k) for k in range(T))
+        want = np.linalg.matrix_power(B, T) @ x0[:, j] + acc @ (p.alpha * a[:, j] * c[:, j])
+        assert np.allclose(s.x[:, j], want, atol=1e-12)
+    assert np.allclose(s.g, a * (s.x - c), atol=1e-12)  # the kept gradient is the one at the current model
+
+
+def test_dpsgd_plain_form_and_mean_descent():
+    """K = 1, eta = 0: x' = M x - alpha g (a non-symmetric M fixes which index of W is summed); the worker
+    mean moves by -alpha times the mean gradient because M is doubly stochastic."""
+    w = inputs.directed_cycle_blend(6, 0.45, 0.35)
+    rng = np.random.default_rng(3)
+    a = rng.uniform(0.5, 2.0, (6, 4))
+    c = rng.standard_normal((6, 4))
+    p = _problem(w, 1, 0.0, 0.07, a, c, 0.2, seed=5)
+    s = orc.init_dpsgd_state(p, rng.standard_normal((6, 4)))
+    for _ in range(4):
+        nxt = orc.dpsgd_step(p, s)
+        assert np.allclose(nxt.x, w.to_dense() @ s.x - 0.07 * s.g, atol=1e-13)
+        assert np.allclose(nxt.x.mean(0), s.x.mean(0) - 0.07 * s.g.mean(0), atol=1e-13)
+        s = nxt
+
+
+def test_dpsgd_average_consensus_with_equal_curvature_is_centralized_gd_on_the_mean():
+    """W = J/n, a_i = a for all workers, noise free: xbar_t = cbar + (1 - alpha a)^t (xbar_0 - cbar), although the
+    workers themselves never agree."""
+    n, m, alpha = 5, 3, 0.1
+    rng = np.random.default_rng(8)
+    a = np.tile(rng.uniform(0.5, 2.0, (1, m)), (n, 1))
+    c = rng.standard_normal((n, m))
+    p = _problem(inputs.average_consensus_matrix(n), 1, 0.0, alpha, a, c, 0.0)
+    x0 = rng.standard_normal((n, m))
+    s = orc.run_dpsgd(p, x0, 9)
+    want = c.mean(0) + (1 - alpha * a[0]) ** 9 * (x0.mean(0) - c.mean(0))
+    assert np.allclose(s.x.mean(0), want, atol=1e-13)
+    assert orc.consensus_error(s.x) > 1e-4  # non-iid data: D-PSGD's workers stay apart at a constant step size
+
+
+def test_dpsgd_fixed_point_is_biased_where_detag_is_not():
+    """The noise-free D-PSGD limit solves (I - P + alpha D_a) x = alpha D_a c per coordinate (library solve); it is
+    not the minimiser of the average objective, which DeTAG reaches on the same problem."""
+    p, w = _small_problem(23, n=8, m=4, K=2, sigma=0.0, alpha=0.05)
+    P = _dense_polynomial(w.to_dense(), p.K, p.eta)
+    a, c = p.a.astype(np.float64), p.c.astype(np.float64)
+    s = orc.run_dpsgd(p, np.zeros((8, 4)), 3000)
+    for j in range(4):
+        want = np.linalg.solve(np.eye(8) - P + p.alpha * np.diag(a[:, j]), p.alpha * a[:, j] * c[:, j])
+        assert np.allclose(s.x[:, j], want, atol=1e-9)
+    xstar = (a * c).sum(0) / a.sum(0)
+    assert np.abs(s.x - xstar[None, :]).max() > 1e-2
+    assert np.allclose(orc.run(p, np.zeros((8, 4)), 3000).x, np.tile(xstar, (8, 1)), atol=1e-9)
+
+
 def test_phase_length_of_theorem_3():
     # sqrt(1 - lambda) = 1/2: R = ln(16) = 2.77 -> 3 rounds; the data-heterogeneity term takes over when it is larger
     assert orc.phase_length(16, 0.75, 0.0, 0.0, 1.0) == 3

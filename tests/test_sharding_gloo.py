@@ -69,3 +69,24 @@ def test_two_gloo_ranks_reproduce_the_single_process_run(tmp_path):
     for q in parts:
         assert float(q["ce"]) == pytest.approx(orc.consensus_error(full.x), rel=1e-12)
         assert float(q["slowest"]) == 11.0
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_is_around():
+    """`python bench.py --gpus 2` with WORLD_SIZE unset must start two ranks itself.  --host-only keeps the run on
+    the CPU: the ranks meet over gloo and reduce the two scalars of the real run through the same helpers."""
+    import json
+    import subprocess
+    import sys
+
+    from conftest import ROOT
+
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--host-only", "--config", "cfg2"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(ln) for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1  # rank 0 alone prints
+    line = lines[0]
+    assert line["host_only"] is True and line["n_gpus"] == 2
+    assert line["slowest"] == 2.0  # MAX over ranks of (1 + rank)
+    assert line["offset_sum"] == float(inputs.CONFIGS["cfg2"].d)  # rank 1's shard starts where rank 0's ends
