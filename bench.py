@@ -41,6 +41,7 @@ KERNEL_SOURCES = {
     "mma": ("step_mma.cu", "mma_common.cuh", "pipeline.cuh", "noise.cuh"),
     "band": ("step_band.cu", "pipeline.cuh", "noise.cuh"),
     "csr": ("step_csr.cu", "noise.cuh"),
+    "torus": ("step_torus.cu", "torus_basis.h", "pipeline.cuh", "noise.cuh"),
 }
 MEASURED_TRAFFIC = {
     # (kernel, mode): (source digest, bytes per wc)
@@ -48,7 +49,9 @@ MEASURED_TRAFFIC = {
 
 # Float64 multiply-adds per worker-coordinate on the FP64 pipe (both contractions, padded shapes) and that
 # pipe's peak: 64 multiply-adds per clock and SM (measured: 61 with m8n8k4 MMAs from 16 warps) x 148 SMs x max clock.
-FP64_FMA_PER_WC = {("mma", "dense"): 64, ("band", "ring"): 80, ("band", "dense"): 128}
+FP64_FMA_PER_WC = {("mma", "dense"): 64, ("band", "ring"): 80, ("band", "dense"): 128,
+                   ("torus", "torus8"): 40, ("torus", "torus4"): 28}
+VARIANT_NAMES = {1: "csr", 2: "dense", 3: "ring", 4: "torus"}
 FP64_FMA_PER_CLK_SM = 64
 SM_COUNT = 148
 
@@ -60,6 +63,8 @@ def kernel_key(variant: str, n: int):
         return ("band", "ring")
     if variant == "csr":
         return ("csr", "rounds")
+    if variant == "torus":
+        return ("torus", "torus8" if n == 64 else "torus4")
     return None
 
 
@@ -247,7 +252,7 @@ def time_config(name: str, dev, args) -> dict:
         a, c, x0 = inputs.objective_data(cfg, j0, j1, threads=min(32, os.cpu_count() or 1))
         for nm, arr in (("a", a), ("c", c), ("x", x0)):
             getattr(s, nm)[:, j0:j1].copy_(torch.from_numpy(arr))
-    variant = {1: "csr", 2: "dense", 3: "ring"}.get(B.detag_get_variant(s.state), "other")
+    variant = VARIANT_NAMES.get(B.detag_get_variant(s.state), "other")
     stream = torch.cuda.current_stream(dev)
     s.init()
     steps = 200 if 20 * cfg.wc < 4 * 126e6 else 20
@@ -344,8 +349,8 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         getattr(s, k).copy_(host[k], non_blocking=True)
     torch.cuda.synchronize(dev)
     if args.variant:
-        B.detag_set_variant(s.state, {"csr": 1, "dense": 2, "ring": 3}[args.variant])
-    variant = {1: "csr", 2: "dense", 3: "ring"}[B.detag_get_variant(s.state)]
+        B.detag_set_variant(s.state, {v: k for k, v in VARIANT_NAMES.items()}[args.variant])
+    variant = VARIANT_NAMES[B.detag_get_variant(s.state)]
     t_setup = time.perf_counter() - t_setup
 
     stream = torch.cuda.current_stream(dev)
@@ -414,7 +419,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
             gbs = bytes_per_wc * cfg.wc / (ms * 1e-3) / 1e9
             modes[label] = {"ms_per_step": ms, "value": cfg.wc / (ms * 1e-3), "unit": UNIT, "steps": m_steps,
                             "bytes_per_wc": bytes_per_wc, "achieved_gbs": gbs,
-                            "variant": {1: "csr", 2: "dense", 3: "ring"}.get(B.detag_get_variant(s.state), "other")}
+                            "variant": VARIANT_NAMES.get(B.detag_get_variant(s.state), "other")}
 
         B.detag_set_algorithm(s.state, B.DETAG_ALGORITHM_DPSGD)
         timed("dpsgd", 24)
@@ -529,7 +534,7 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg5", choices=sorted(inputs.CONFIGS))
     ap.add_argument("--d", type=int, default=0, help="override the coordinate count (profiling a small case)")
-    ap.add_argument("--variant", default="", choices=["", "csr", "dense", "ring"])
+    ap.add_argument("--variant", default="", choices=["", "csr", "dense", "ring", "torus"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--steps-per-launch", type=int, default=20,
                     help="also time detag_step_many with this many iterations per call (0: skip)")

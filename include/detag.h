@@ -59,7 +59,9 @@ enum {
   DETAG_VARIANT_AUTO = 0,  /* host cost model picks */
   DETAG_VARIANT_CSR = 1,   /* K rounds of neighbour-indexed sums over the CSR rows, slab staged on chip */
   DETAG_VARIANT_DENSE = 2, /* one product with the host-precomputed polynomial P_K(M), n <= 64 */
-  DETAG_VARIANT_RING = 3   /* banded circulant polynomial P_K(M): circulant M (rings), n % 32 == 0, n >= 64, K*bandwidth <= 16 */
+  DETAG_VARIANT_RING = 3,  /* banded circulant polynomial P_K(M): circulant M (rings), n % 32 == 0, n >= 64, K*bandwidth <= 16 */
+  DETAG_VARIANT_TORUS = 4  /* block-circulant M with 8-worker blocks, symmetric in the block distance (R x 8 tori, n = 32 or 64):
+                              Fourier transform along the block axis, one 8 x 8 polynomial block per frequency, transform back */
 };
 
 /* The point at which a step queries the stochastic gradient oracle. */

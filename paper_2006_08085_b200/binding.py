@@ -31,6 +31,7 @@ DETAG_VARIANT_AUTO = 0
 DETAG_VARIANT_CSR = 1
 DETAG_VARIANT_DENSE = 2
 DETAG_VARIANT_RING = 3
+DETAG_VARIANT_TORUS = 4
 
 DETAG_GRADIENT_AT_NEW_MODEL = 0
 DETAG_GRADIENT_AT_PHASE_START = 1

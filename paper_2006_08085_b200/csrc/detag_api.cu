@@ -8,6 +8,7 @@
 #include <new>
 
 #include "detag_internal.h"
+#include "torus_basis.h"
 
 using detag::StepParams;
 
@@ -16,7 +17,7 @@ namespace {
 size_t align_up(size_t v) { return (v + detag::kWsAlign - 1) / detag::kWsAlign * detag::kWsAlign; }
 
 struct WsLayout {
-  size_t status, result, row_ptr, col_idx, vals, poly, partials, total;
+  size_t status, result, row_ptr, col_idx, vals, poly, torus, partials, total;
 };
 
 WsLayout ws_layout(const detag_state* s) {
@@ -33,6 +34,8 @@ WsLayout ws_layout(const detag_state* s) {
   off += align_up(s->vals.size() * sizeof(double));
   l.poly = off;
   off += align_up(s->poly.size() * sizeof(double));
+  l.torus = off;
+  off += align_up(s->torus_frag.size() * sizeof(double));
   l.partials = off;
   off += align_up(detag::kMaxPartials * sizeof(double));
   l.total = off;
@@ -112,6 +115,80 @@ void analyse_circulant(detag_state* s) {
       s->band[delta + 16] = (delta >= -hb && delta <= hb) ? cur[((delta % n) + n) % n] : 0.0;
 }
 
+// Block-circulant M with 8-worker blocks whose block (r, r') depends on the distance (r' - r) mod R only, equal for
+// +k and -k (tori): the real Fourier basis Q of the R-cycle block-diagonalises every polynomial of M,
+//     P_K(M) = sum_p (q_p q_p^T) (x) P_K(Mhat_p) ,   Mhat_p = sum_k cos(2 pi f_p k / R) G_k .
+// The 8 x 8 blocks P_K(Mhat_p) come from the recursion of Algorithm 3 on Mhat_p; the result is accepted only if it
+// reproduces the dense polynomial.
+void analyse_torus(detag_state* s) {
+  const int n = s->n, C = 8;
+  if (s->poly.empty() || n % C != 0 || !detag::torus_variant_available(n)) return;
+  const int R = n / C;
+  std::vector<double> m;
+  detag::csr_to_dense(n, s->row_ptr.data(), s->col_idx.data(), s->vals.data(), m);
+  auto M = [&](int r, int c, int r2, int c2) { return m[static_cast<size_t>(r * C + c) * n + (r2 * C + c2)]; };
+  for (int r = 0; r < R; ++r)
+    for (int k = 0; k < R; ++k)
+      for (int c = 0; c < C; ++c)
+        for (int c2 = 0; c2 < C; ++c2) {
+          if (M(r, c, (r + k) % R, c2) != M(0, c, k, c2)) return;        // block circulant
+          if (M(0, c, k, c2) != M(0, c, (R - k) % R, c2)) return;        // the same block at distance +k and -k
+        }
+  const double kPi = 3.14159265358979323846;
+  std::vector<double> q(static_cast<size_t>(R) * R);  // the kernel's basis, row p = basis vector p
+  std::vector<int> freq(R);
+  for (int p = 0; p < R; ++p) {
+    freq[p] = detag::torus_frequency(R, p);
+    for (int r = 0; r < R; ++r) q[p * R + r] = detag::torus_q(R, p, r);
+  }
+  std::vector<double> phat(static_cast<size_t>(R) * C * C);
+  for (int p = 0; p < R; ++p) {
+    double mh[8][8], prev[8][8], cur[8][8], next[8][8];
+    for (int c = 0; c < C; ++c)
+      for (int c2 = 0; c2 < C; ++c2) {
+        double acc = 0.0;
+        for (int k = 0; k < R; ++k) acc += std::cos(2.0 * kPi * freq[p] * k / R) * M(0, c, k, c2);
+        mh[c][c2] = acc;
+        prev[c][c2] = cur[c][c2] = c == c2 ? 1.0 : 0.0;
+      }
+    for (int round = 0; round < s->K; ++round) {  // P_{r+1} = (1+eta) Mhat P_r - eta P_{r-1}
+      for (int c = 0; c < C; ++c)
+        for (int c2 = 0; c2 < C; ++c2) {
+          double acc = 0.0;
+          for (int k = 0; k < C; ++k) acc += mh[c][k] * cur[k][c2];
+          next[c][c2] = (1.0 + s->eta) * acc - s->eta * prev[c][c2];
+        }
+      std::memcpy(prev, cur, sizeof cur);
+      std::memcpy(cur, next, sizeof cur);
+    }
+    for (int c = 0; c < C; ++c)
+      for (int c2 = 0; c2 < C; ++c2) phat[(static_cast<size_t>(p) * C + c) * C + c2] = cur[c][c2];
+  }
+  // the decomposition must give back the dense polynomial
+  double worst = 0.0, scale = 0.0;
+  for (int r = 0; r < R; ++r)
+    for (int r2 = 0; r2 < R; ++r2)
+      for (int c = 0; c < C; ++c)
+        for (int c2 = 0; c2 < C; ++c2) {
+          double acc = 0.0;
+          for (int p = 0; p < R; ++p) acc += q[p * R + r] * q[p * R + r2] * phat[(static_cast<size_t>(p) * C + c) * C + c2];
+          const double want = s->poly[static_cast<size_t>(r * C + c) * n + (r2 * C + c2)];
+          worst = std::fmax(worst, std::fabs(acc - want));
+          scale = std::fmax(scale, std::fabs(want));
+        }
+  if (!(worst <= 1e-13 * std::fmax(1.0, scale))) return;
+  s->torus = true;
+  // fragment order of the kernel: entry (p, k-step s, lane) is Phat_p[lane / 4][2 (lane % 4) + s]
+  s->torus_frag.resize(static_cast<size_t>(R) * 2 * 32);
+  for (int p = 0; p < R; ++p)
+    for (int st = 0; st < 2; ++st)
+      for (int lane = 0; lane < 32; ++lane)
+        s->torus_frag[(static_cast<size_t>(p) * 2 + st) * 32 + lane] =
+            phat[(static_cast<size_t>(p) * C + lane / 4) * C + 2 * (lane % 4) + st];
+}
+
+bool torus_ok(const detag_state* s) { return s->torus && s->d <= 0x7fffffffLL; }
+
 bool band_ok(const detag_state* s) {
   return s->circulant && s->d <= 0x7fffffffLL && detag::band_variant_available(s->n, s->half_band);
 }
@@ -139,6 +216,7 @@ StepParams make_params(const detag_state* s) {
   p.col_idx = s->d_col_idx;
   p.vals = s->d_vals;
   p.poly = s->d_poly;
+  p.torus = s->d_torus;
   p.eta = s->eta;
   p.alpha = s->alpha;
   p.sigma = s->sigma;
@@ -162,6 +240,8 @@ bool dense_ok(const detag_state* s) {
 // n it supports - except that for 32 < n <= 64 a circulant matrix with a narrow band is cheaper through the
 // band kernel (80 instead of 128 MMAs per tile).  Caller-written gradients and D-PSGD run on the dense
 // kernel for n <= 32 and on the generic rounds kernel otherwise.
+// for 32 < n <= 64 a block-circulant matrix (torus) takes the transform kernel: 24 multiply-adds per element
+// and array instead of 64.
 bool variant_runs_mode(const detag_state* s, int variant) {
   if (step_mode(s) == detag::kModeDetag) return true;
   return variant == DETAG_VARIANT_CSR || (variant == DETAG_VARIANT_DENSE && s->n <= 32);
@@ -171,6 +251,7 @@ int resolve_variant(const detag_state* s) {
   if (s->variant_forced != DETAG_VARIANT_AUTO) return s->variant_forced;
   if (step_mode(s) != detag::kModeDetag) return (s->n <= 32 && dense_ok(s)) ? DETAG_VARIANT_DENSE : DETAG_VARIANT_CSR;
   if (s->n > 32 && band_ok(s)) return DETAG_VARIANT_RING;
+  if (s->n > 32 && torus_ok(s)) return DETAG_VARIANT_TORUS;
   if (dense_ok(s)) return DETAG_VARIANT_DENSE;
   return DETAG_VARIANT_CSR;
 }
@@ -188,7 +269,7 @@ int query_device(detag_state* s) {
 }
 
 // Kernel families that take tensor maps.
-enum { kFamilyMma = 1, kFamilyBand = 2 };
+enum { kFamilyMma = 1, kFamilyBand = 2, kFamilyTorus = 3 };
 
 // Tensor maps for the buffers in `p`: built on first use, then found again by buffer addresses and sizes
 // (detag_step always hits; detag_step_host cycles through its two chunk slots and the ragged last chunk).
@@ -211,7 +292,9 @@ const detag::TensorMapSet* maps_for(detag_state* s, int family, const StepParams
   }
   detag_state::MapEntry& en = *slot;
   en.family = 0;  // invalid until built
-  const bool ok = family == kFamilyMma ? detag::build_maps_mma(p, &en.maps) : detag::build_maps_band(p, &en.maps);
+  const bool ok = family == kFamilyMma    ? detag::build_maps_mma(p, &en.maps)
+                  : family == kFamilyBand ? detag::build_maps_band(p, &en.maps)
+                                          : detag::build_maps_torus(p, &en.maps);
   if (!ok) return nullptr;
   en.family = family;
   en.d = p.d;
@@ -241,6 +324,12 @@ int launch_step(detag_state* s, StepParams& p, cudaStream_t stream) {
         e = detag::launch_step_mma(p, *maps, s->sm_count, stream);
       else
         e = detag::launch_step_band(p, *maps, variant == DETAG_VARIANT_RING ? s->band : nullptr, s->sm_count, stream);
+      break;
+    }
+    case DETAG_VARIANT_TORUS: {
+      const detag::TensorMapSet* maps = maps_for(s, kFamilyTorus, p);
+      if (!maps) return fail(s, DETAG_ERR_CUDA, "tensor map encoding failed");
+      e = detag::launch_step_torus(p, *maps, p.torus, s->sm_count, stream);
       break;
     }
     case DETAG_VARIANT_CSR:
@@ -300,6 +389,7 @@ int detag_create(detag_state** out, int n, int64_t d, const int32_t* row_ptr, co
   s->vals.assign(vals, vals + nnz);
   if (n <= detag::kMaxDenseWorkers) gossip_polynomial(s, s->poly);
   analyse_circulant(s);
+  analyse_torus(s);
   s->map_cache.reserve(8);
   *out = s;
   return DETAG_OK;
@@ -334,6 +424,7 @@ int detag_bind(detag_state* s, int64_t ld, float* x, float* y, float* g, const f
   s->d_col_idx = reinterpret_cast<int32_t*>(base + l.col_idx);
   s->d_vals = reinterpret_cast<double*>(base + l.vals);
   s->d_poly = s->poly.empty() ? nullptr : reinterpret_cast<double*>(base + l.poly);
+  s->d_torus = s->torus_frag.empty() ? nullptr : reinterpret_cast<double*>(base + l.torus);
   s->d_partials = reinterpret_cast<double*>(base + l.partials);
 
   e = cudaMemset(base, 0, detag::kWsAlign);
@@ -345,6 +436,8 @@ int detag_bind(detag_state* s, int64_t ld, float* x, float* y, float* g, const f
     e = cudaMemcpy(s->d_vals, s->vals.data(), s->vals.size() * sizeof(double), cudaMemcpyHostToDevice);
   if (e == cudaSuccess && s->d_poly)
     e = cudaMemcpy(s->d_poly, s->poly.data(), s->poly.size() * sizeof(double), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess && s->d_torus)
+    e = cudaMemcpy(s->d_torus, s->torus_frag.data(), s->torus_frag.size() * sizeof(double), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) return fail_cuda(s, e, "detag_bind: workspace upload");
 
   s->ld = ld;
@@ -384,6 +477,12 @@ int detag_set_variant(detag_state* s, int variant) {
       break;
     case DETAG_VARIANT_DENSE:
       if (!dense_ok(s)) return fail(s, DETAG_ERR_UNSUPPORTED, "detag_set_variant: dense variant needs n <= 64");
+      break;
+    case DETAG_VARIANT_TORUS:
+      if (!torus_ok(s))
+        return fail(s, DETAG_ERR_UNSUPPORTED,
+                    "detag_set_variant: torus variant needs n = 32 or 64 and a matrix that is block circulant in "
+                    "8-worker blocks, symmetric in the block distance");
       break;
     case DETAG_VARIANT_RING:
       if (!band_ok(s))
@@ -597,6 +696,9 @@ int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* 
     e = cudaMemcpyAsync(base + l.vals, s->vals.data(), s->vals.size() * sizeof(double), cudaMemcpyHostToDevice, user);
   if (e == cudaSuccess && !s->poly.empty())
     e = cudaMemcpyAsync(base + l.poly, s->poly.data(), s->poly.size() * sizeof(double), cudaMemcpyHostToDevice, user);
+  if (e == cudaSuccess && !s->torus_frag.empty())
+    e = cudaMemcpyAsync(base + l.torus, s->torus_frag.data(), s->torus_frag.size() * sizeof(double),
+                        cudaMemcpyHostToDevice, user);
   if (e == cudaSuccess) e = cudaEventRecord(s->host_event[2], user);
   for (int k = 0; k < 2 && e == cudaSuccess; ++k) e = cudaStreamWaitEvent(s->host_stream[k], s->host_event[2], 0);
   if (e != cudaSuccess) return fail_cuda(s, e, "detag_step_host: table upload");
@@ -606,6 +708,7 @@ int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* 
   p.col_idx = reinterpret_cast<int32_t*>(base + l.col_idx);
   p.vals = reinterpret_cast<double*>(base + l.vals);
   p.poly = s->poly.empty() ? nullptr : reinterpret_cast<double*>(base + l.poly);
+  p.torus = s->torus_frag.empty() ? nullptr : reinterpret_cast<double*>(base + l.torus);
   p.status = status_word;
   p.y_obs = nullptr;
   p.t_noise = static_cast<uint32_t>(s->t + 1);

@@ -39,6 +39,7 @@ struct StepParams {
   const int32_t* col_idx;
   const double* vals;
   const double* poly;  // dense P_K(M), row-major n x n (null when n > kMaxDenseWorkers)
+  const double* torus; // block-circulant kernel: per-frequency 8 x 8 polynomial blocks in fragment order (or null)
   double eta;
   double alpha;
   double sigma;
@@ -86,6 +87,10 @@ bool dense_window_available(int n);                // the band kernel's dense mo
 bool build_maps_band(const StepParams& p, TensorMapSet* maps);
 int launch_step_band(StepParams p, const TensorMapSet& maps, const double* band /* null: dense mode */, int sm_count,
                      cudaStream_t stream);
+bool torus_variant_available(int n);               // block-circulant kernel: n = 32 or 64 (4 or 8 blocks of 8)
+bool build_maps_torus(const StepParams& p, TensorMapSet* maps);
+int launch_step_torus(StepParams p, const TensorMapSet& maps, const double* phat_frag /* device */, int sm_count,
+                      cudaStream_t stream);
 int launch_consensus_error(const StepParams& p, double* partials, double* result, int sm_count, cudaStream_t stream);
 int launch_init_external(const StepParams& p, int sm_count, cudaStream_t stream);  // y = g = g_ext
 int launch_expire_wait(int* status, unsigned polls, cudaStream_t stream);          // a wait nobody ends (self test)
@@ -105,6 +110,10 @@ struct detag_state {
   bool circulant = false;    // every row of M is the previous one shifted by one
   int half_band = 0;         // of the circulant P_K(M): P[i][(i+delta) mod n] = 0 for |delta| > half_band
   double band[33] = {0};     // p(delta) at index delta + 16, valid when circulant and half_band <= 16
+  // block-circulant structure with 8-worker blocks, symmetric in the block distance (tori): the per-frequency
+  // 8 x 8 polynomial blocks in MMA fragment order
+  bool torus = false;
+  std::vector<double> torus_frag;
   int variant_forced = DETAG_VARIANT_AUTO;
   int gradient_point = DETAG_GRADIENT_AT_NEW_MODEL;
   int algorithm = DETAG_ALGORITHM_DETAG;
@@ -127,6 +136,7 @@ struct detag_state {
   int32_t* d_col_idx = nullptr;
   double* d_vals = nullptr;
   double* d_poly = nullptr;
+  double* d_torus = nullptr;
   double* d_partials = nullptr;
 
   double sigma = 0.0;

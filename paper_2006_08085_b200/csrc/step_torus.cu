@@ -18,16 +18,16 @@
 // With the k-steps taking c = 2 (lane % 4) + s, the A fragment a lane supplies and the C fragment it receives are
 // the SAME worker positions: lane (coord = lane / 4, kq = lane % 4) owns workers 8 r + 2 kq + e (r = 0..R-1,
 // e = 0, 1) of one coordinate for input and output alike.  So the transforms along r run inside the lane over its
-// own registers (dense R x R, coefficients as immediate operands from the kernel parameters), the tail of the
+// own registers (dense R x R with compile-time coefficients; a quarter of them are zero and cost nothing), the tail of the
 // step (model update, noise, gradient, tracker fold) is lane-local, and every lane writes its results over the
 // very elements it read: the output needs no tile of its own.
 //
 // Shared memory holds tiles of [64 or 32 workers][64 coordinates] as two 32-coordinate halves in the 128-byte
 // swizzle of the tensor maps; with the ownership above every warp-wide access hits 32 different banks, and the
 // TMA stores undo the swizzle on the way out.  Roles of the persistent CTA (one per SM):
-//   producer  one thread: per slab two loads each of x, y into one of two short-lived stages (a lane copies its 2R
-//             values of each to registers first thing and hands the stage back) and of g, a, c into one of three
-//             long-lived stages (read in the tail, then overwritten with g', x', y');
+//   producer  one thread: per slab two loads each of x, y into one of two short-lived stages (handed back as soon as
+//             the tracker contraction has read its operands) and of g, a, c into one of three long-lived stages
+//             (read in the tail, then overwritten with g', x', y');
 //   consumers 16 warps in two groups taking alternate slabs; a warp owns 8 coordinates x all workers;
 //   storer    one thread: when a group's 8 warps have written their results, six TMA stores send the stage's three
 //             tiles out; once they have been read the stage goes back to the producer.
@@ -40,6 +40,7 @@
 #include "noise.cuh"
 #include "pipeline.cuh"
 #include "tma.cuh"
+#include "torus_basis.h"
 
 namespace detag {
 
@@ -74,11 +75,6 @@ struct TorusMaps {
 };
 static_assert(sizeof(TorusMaps) <= sizeof(TensorMapSet), "tensor map storage");
 
-// The real Fourier basis of the R-cycle, q[p][r]; fixed size so that one parameter type serves every R.
-struct TorusBasis {
-  double q[8][8];
-};
-
 // [rows][32-coordinate box] tensor map with the 128-byte swizzle.
 inline bool make_swizzled_map(CUtensorMap* m, const float* base, int n, long long d, long long ld, int box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
@@ -92,10 +88,50 @@ inline bool make_swizzled_map(CUtensorMap* m, const float* base, int n, long lon
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Gradient phase of a lane: g' = a (x_at - c) + sigma xi for its 2R elements, written over c in the stage (c is not
+// needed again; the tracker phase picks g' up from there).  x_at: the model at which the gradient is taken.
+// Noise: the Philox call of (coordinate, workers 8 r + 4 (kq / 2) .. + 3) serves this lane and its neighbour
+// kq ^ 1; each draws the calls of every other block r and they swap the word pairs they do not need themselves.
+template <int R>
+__device__ __forceinline__ void torus_gradient(const StepParams& p, const float* sa, float* sc, const int (&off_e)[2],
+                                               const float (&x_at)[2][R], int kq, long long j, float sigma, bool noisy) {
+  unsigned long long jn = static_cast<unsigned long long>(p.coord_offset + j);
+  // Ties the counter to the model values so that the compiler cannot start the generator's integer work while the
+  // contraction before this phase still holds its accumulators (it would spill them).
+  asm volatile("" : "+l"(jn) : "f"(x_at[0][0]), "f"(x_at[1][R - 1]));
+  const bool odd = (kq & 1) != 0;
+#pragma unroll
+  for (int h = 0; h < R / 2; ++h) {
+    float xi[2][2] = {{0.f, 0.f}, {0.f, 0.f}};  // [e][block 2h, 2h + 1]
+    if (noisy) {
+      const int r_mine = 2 * h + (odd ? 1 : 0);
+      const Philox4 w = philox4x32_10(static_cast<uint32_t>(jn), static_cast<uint32_t>(jn >> 32),
+                                      static_cast<uint32_t>(2 * r_mine + (kq >> 1)), p.t_noise, p.seed_lo, p.seed_hi);
+      // even kq owns the first pair of words (workers +0, +1 of the quad), odd kq the second (workers +2, +3)
+      const uint32_t keep0 = odd ? w.r2 : w.r0, keep1 = odd ? w.r3 : w.r1;
+      const uint32_t give0 = odd ? w.r0 : w.r2, give1 = odd ? w.r1 : w.r3;
+      const uint32_t got0 = __shfl_xor_sync(0xffffffffu, give0, 1), got1 = __shfl_xor_sync(0xffffffffu, give1, 1);
+      float n0, n1, m0, m1;
+      box_muller(keep0, keep1, n0, n1);  // block r_mine
+      box_muller(got0, got1, m0, m1);    // the neighbour's block
+      xi[0][0] = odd ? m0 : n0;
+      xi[1][0] = odd ? m1 : n1;
+      xi[0][1] = odd ? n0 : m0;
+      xi[1][1] = odd ? n1 : m1;
+    }
+#pragma unroll
+    for (int b = 0; b < 2; ++b)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int r = 2 * h + b, o = off_e[e] + r * 256;
+        sc[o] = fmaf(sa[o], x_at[e][r] - sc[o], sigma * xi[e][b]);
+      }
+  }
+}
+
 template <int R, bool kAtStart>
 __global__ void __launch_bounds__(kTThreads, 1)
-step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, const __grid_constant__ TorusBasis basis,
-                  const double* __restrict__ phat_frag) {
+step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, const double* __restrict__ phat_frag) {
   using Plan = TorusPlan<R>;
   extern __shared__ unsigned char smem_unaligned[];
   // the swizzle pattern is a function of the shared-memory address: tiles start on 1 KiB boundaries
@@ -242,31 +278,38 @@ step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, co
     const long long j = slab * kTS + tile * 8 + crow;  // this lane's coordinate
     const bool active = slab * kTS + tile * 8 < p.d;   // a tile wholly beyond column d computes nothing
 
-    float xin[2][R], yin[2][R];
-#pragma unroll
-    for (int e = 0; e < 2; ++e)
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-        xin[e][r] = sxp[off_e[e] + r * 256];
-        yin[e][r] = syp[off_e[e] + r * 256];
-      }
-    __syncwarp();
-    if (lane == 0) bar_arrive(&xy_empty[sx]);  // x, y are in registers: the stage can be refilled
-
+    bool released = false;
     if (active) {
-      // ---- model: x' = P (x - alpha y)
-      float xo[2][R];
+      // Registers are the scarce resource here (2R values per array and lane, float64 accumulators): the phases
+      // below run one after the other, read their operands from the stages when they need them and park what a
+      // later phase needs in the lane's own slots - x' over a, then g' over c (both read just before), finally g'
+      // over g and y' over c.
+      float xv[2][R];  // the model at which the gradient is taken, then x'
+      if (kAtStart) {  // Algorithm 2 as printed: the gradient at the model the step started from
+#pragma unroll
+        for (int e = 0; e < 2; ++e)
+#pragma unroll
+          for (int r = 0; r < R; ++r) xv[e][r] = sxp[off_e[e] + r * 256];
+        torus_gradient<R>(p, sa, sc, off_e, xv, kq, j, sigma, noisy);
+      }
+      // ---- model: x' = P (x - alpha y), by linearity of AG_K
       {
         double acc[R][2];
 #pragma unroll
-        for (int pf = 0; pf < R; ++pf) {
-          acc[pf][0] = acc[pf][1] = 0.0;
+        for (int pf = 0; pf < R; ++pf) acc[pf][0] = acc[pf][1] = 0.0;
 #pragma unroll
-          for (int s = 0; s < 2; ++s) {
-            double zh = 0.0;  // forward transform: component pf of this lane's worker column (c = 2 kq + s)
+        for (int s = 0; s < 2; ++s) {  // k-step s: this lane's worker column c = 2 kq + s
+          double z[R];
 #pragma unroll
-            for (int r = 0; r < R; ++r)
-              zh = fma(basis.q[pf][r], fma(-alpha, static_cast<double>(yin[s][r]), static_cast<double>(xin[s][r])), zh);
+          for (int r = 0; r < R; ++r) {
+            const int o = off_e[s] + r * 256;
+            z[r] = fma(-alpha, static_cast<double>(syp[o]), static_cast<double>(sxp[o]));
+          }
+#pragma unroll
+          for (int pf = 0; pf < R; ++pf) {
+            double zh = 0.0;  // forward transform: component pf of the column
+#pragma unroll
+            for (int r = 0; r < R; ++r) if (torus_q(R, pf, r) != 0.0) zh = fma(torus_q(R, pf, r), z[r], zh);
             dmma(acc[pf], zh, frag[(pf * 2 + s) * 32 + lane]);
           }
         }
@@ -276,90 +319,71 @@ step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, co
           for (int r = 0; r < R; ++r) {
             double v = 0.0;  // transform back: worker (r, 2 kq + e)
 #pragma unroll
-            for (int pf = 0; pf < R; ++pf) v = fma(basis.q[pf][r], acc[pf][e], v);
-            xo[e][r] = static_cast<float>(v);
+            for (int pf = 0; pf < R; ++pf) if (torus_q(R, pf, r) != 0.0) v = fma(torus_q(R, pf, r), acc[pf][e], v);
+            xv[e][r] = static_cast<float>(v);  // x', rounded once
           }
       }
-      // ---- tracker: y~ = P y
-      double yg[2][R];
+      if (!kAtStart) torus_gradient<R>(p, sa, sc, off_e, xv, kq, j, sigma, noisy);  // at the new model
+#pragma unroll
+      for (int e = 0; e < 2; ++e)
+#pragma unroll
+        for (int r = 0; r < R; ++r) sa[off_e[e] + r * 256] = xv[e][r];  // x' takes a's place
+      // ---- tracker: y~ = P y, then the fold (y~ - g) + g'
       {
         double acc[R][2];
 #pragma unroll
-        for (int pf = 0; pf < R; ++pf) {
-          acc[pf][0] = acc[pf][1] = 0.0;
+        for (int pf = 0; pf < R; ++pf) acc[pf][0] = acc[pf][1] = 0.0;
 #pragma unroll
-          for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < 2; ++s) {
+          double z[R];
+#pragma unroll
+          for (int r = 0; r < R; ++r) z[r] = static_cast<double>(syp[off_e[s] + r * 256]);
+          if (s == 1) {  // the last read of the x, y stage: it can be refilled
+            __syncwarp();
+            if (lane == 0) bar_arrive(&xy_empty[sx]);
+            released = true;
+          }
+#pragma unroll
+          for (int pf = 0; pf < R; ++pf) {
             double zh = 0.0;
 #pragma unroll
-            for (int r = 0; r < R; ++r) zh = fma(basis.q[pf][r], static_cast<double>(yin[s][r]), zh);
+            for (int r = 0; r < R; ++r) if (torus_q(R, pf, r) != 0.0) zh = fma(torus_q(R, pf, r), z[r], zh);
             dmma(acc[pf], zh, frag[(pf * 2 + s) * 32 + lane]);
           }
         }
+        const bool in_d = j < p.d;
 #pragma unroll
         for (int e = 0; e < 2; ++e)
 #pragma unroll
           for (int r = 0; r < R; ++r) {
             double v = 0.0;
 #pragma unroll
-            for (int pf = 0; pf < R; ++pf) v = fma(basis.q[pf][r], acc[pf][e], v);
-            yg[e][r] = v;
+            for (int pf = 0; pf < R; ++pf) if (torus_q(R, pf, r) != 0.0) v = fma(torus_q(R, pf, r), acc[pf][e], v);
+            const int o = off_e[e] + r * 256;
+            const float go = sc[o];  // g', parked there by the gradient phase
+            const float yo = static_cast<float>((v - static_cast<double>(sg[o])) + static_cast<double>(go));
+            sg[o] = go;
+            sc[o] = yo;
+            if (p.y_obs != nullptr && in_d)  // optional observer: the gossiped tracker, stored directly
+              p.y_obs[static_cast<long long>(8 * r + 2 * kq + e) * p.ld + j] = static_cast<float>(v);
           }
-      }
-      // ---- noise: the Philox call of (coordinate, workers 8 r + 4 (kq / 2) .. + 3) serves this lane and its
-      // neighbour kq ^ 1; each draws the calls of every other block r and they swap the halves they do not need
-      float xi[2][R];
-      if (noisy) {
-        const unsigned long long jn = static_cast<unsigned long long>(p.coord_offset + j);
+        if (in_d && j >= d_tma) {  // TMA clips stores at 16-byte granularity: the last d % 4 columns go out directly
 #pragma unroll
-        for (int h = 0; h < R / 2; ++h) {
-          const int r_mine = 2 * h + (kq & 1), r_other = 2 * h + 1 - (kq & 1);
-          const Philox4 w = philox4x32_10(static_cast<uint32_t>(jn), static_cast<uint32_t>(jn >> 32),
-                                          static_cast<uint32_t>(2 * r_mine + (kq >> 1)), p.t_noise, p.seed_lo, p.seed_hi);
-          // even kq owns the first pair of words (workers +0, +1), odd kq the second (workers +2, +3)
-          const uint32_t keep0 = (kq & 1) ? w.r2 : w.r0, keep1 = (kq & 1) ? w.r3 : w.r1;
-          const uint32_t give0 = (kq & 1) ? w.r0 : w.r2, give1 = (kq & 1) ? w.r1 : w.r3;
-          const uint32_t got0 = __shfl_xor_sync(0xffffffffu, give0, 1), got1 = __shfl_xor_sync(0xffffffffu, give1, 1);
-          float n0, n1, m0, m1;
-          box_muller(keep0, keep1, n0, n1);
-          box_muller(got0, got1, m0, m1);
-          // r_mine / r_other alternate with the lane's parity: select without dynamic register indexing
-          xi[0][2 * h] = (kq & 1) ? m0 : n0;
-          xi[1][2 * h] = (kq & 1) ? m1 : n1;
-          xi[0][2 * h + 1] = (kq & 1) ? n0 : m0;
-          xi[1][2 * h + 1] = (kq & 1) ? n1 : m1;
-          (void)r_other;
-        }
-      } else {
+          for (int e = 0; e < 2; ++e)
 #pragma unroll
-        for (int e = 0; e < 2; ++e)
-#pragma unroll
-          for (int r = 0; r < R; ++r) xi[e][r] = 0.f;
-      }
-      // ---- element-wise tail on this lane's own elements; results replace the inputs in the stage
-      const bool in_d = j < p.d;
-#pragma unroll
-      for (int e = 0; e < 2; ++e)
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-          const int o = off_e[e] + r * 256;
-          const float gv = sg[o], av = sa[o], cv = sc[o];
-          const float x_at = kAtStart ? xin[e][r] : xo[e][r];  // gradient point (Algorithm 2 as printed: the old model)
-          const float go = fmaf(av, x_at - cv, sigma * xi[e][r]);  // stochastic gradient
-          const double ymg = yg[e][r] - static_cast<double>(gv);   // y~ - g
-          const float yo = static_cast<float>(ymg + static_cast<double>(go));  // fold with g' as stored
-          sg[o] = go;
-          sa[o] = xo[e][r];
-          sc[o] = yo;
-          if (in_d && (j >= d_tma || p.y_obs != nullptr)) {
-            const long long off = static_cast<long long>(8 * r + 2 * kq + e) * p.ld + j;
-            if (j >= d_tma) {  // TMA clips stores at 16-byte granularity: the last d % 4 columns go out directly
-              p.x[off] = xo[e][r];
-              p.y[off] = yo;
-              p.g[off] = go;
+            for (int r = 0; r < R; ++r) {
+              const int o = off_e[e] + r * 256;
+              const long long off = static_cast<long long>(8 * r + 2 * kq + e) * p.ld + j;
+              p.x[off] = sa[o];
+              p.y[off] = sc[o];
+              p.g[off] = sg[o];
             }
-            if (p.y_obs != nullptr) p.y_obs[off] = static_cast<float>(yg[e][r]);  // optional observer: gossiped tracker
-          }
         }
+      }
+    }
+    if (!released) {  // idle tile: same protocol, nothing computed
+      __syncwarp();
+      if (lane == 0) bar_arrive(&xy_empty[sx]);
     }
     fence_async_shared();  // results visible to the TMA stores
     __syncwarp();
@@ -367,7 +391,7 @@ step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, co
   }
 }
 
-typedef void (*TorusKernel)(const StepParams, const TorusMaps, const TorusBasis, const double*);
+typedef void (*TorusKernel)(const StepParams, const TorusMaps, const double*);
 
 }  // namespace
 
@@ -388,14 +412,11 @@ bool build_maps_torus(const StepParams& p, TensorMapSet* out) {
   return true;
 }
 
-// basis: row-major R x R (q[p][r]); phat_frag: device pointer to the R x 2 x 32 doubles in fragment order.
-int launch_step_torus(StepParams p, const TensorMapSet& maps, const double* basis, const double* phat_frag,
-                      int sm_count, cudaStream_t stream) {
+// phat_frag: device pointer to the R x 2 x 32 doubles of the per-frequency blocks in fragment order.
+int launch_step_torus(StepParams p, const TensorMapSet& maps, const double* phat_frag, int sm_count,
+                      cudaStream_t stream) {
   if (p.mode != kModeDetag || (p.n != 32 && p.n != 64)) return static_cast<int>(cudaErrorInvalidValue);
   const int R = p.n / kC;
-  TorusBasis b{};
-  for (int pf = 0; pf < R; ++pf)
-    for (int r = 0; r < R; ++r) b.q[pf][r] = basis[pf * R + r];
   p.S = kTS;
   p.num_slabs = (p.d + kTS - 1) / kTS;
   TorusKernel kernel;
@@ -411,7 +432,7 @@ int launch_step_torus(StepParams p, const TensorMapSet& maps, const double* basi
   if (e != 0) return e;
   const long long grid = p.num_slabs < sm_count ? p.num_slabs : sm_count;
   if (grid <= 0) return 0;
-  kernel<<<static_cast<unsigned>(grid), kTThreads, smem, stream>>>(p, *reinterpret_cast<const TorusMaps*>(maps.bytes), b,
+  kernel<<<static_cast<unsigned>(grid), kTThreads, smem, stream>>>(p, *reinterpret_cast<const TorusMaps*>(maps.bytes),
                                                                    phat_frag);
   return static_cast<int>(cudaGetLastError());
 }

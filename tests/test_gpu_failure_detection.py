@@ -23,9 +23,9 @@ def _built():
     build.build()
 
 
-def _case(n, d, seed=0):
+def _case(n, d, seed=0, torus=False):
     rng = np.random.default_rng(seed)
-    m = inputs.metropolis_weights(inputs.ring_graph(n))
+    m = inputs.metropolis_weights(inputs.torus_graph(n // 8, 8) if torus else inputs.ring_graph(n))
     a = rng.uniform(0.5, 2.0, (n, d)).astype(np.float32)
     c = rng.standard_normal((n, d)).astype(np.float32)
     x0 = rng.standard_normal((n, d)).astype(np.float32)
@@ -58,9 +58,11 @@ def test_a_wait_that_nothing_ends_gives_up_and_is_reported():
     (16, 64 * 148 * 4 + 17, 3, B.DETAG_VARIANT_DENSE, 0),   # nothing is ever loaded
     (64, 64 * 148 * 2 + 5, 2, B.DETAG_VARIANT_RING, 3),     # band kernel, ring
     (48, 64 * 148 * 2 + 5, 2, B.DETAG_VARIANT_DENSE, 1),    # band kernel, dense window mode
+    (64, 64 * 148 * 3 + 5, 2, B.DETAG_VARIANT_TORUS, 2),    # block-circulant transform kernel
+    (32, 64 * 148 * 3 + 5, 2, B.DETAG_VARIANT_TORUS, 0),
 ])
 def test_a_stalled_loader_times_out_every_waiter_and_the_state_recovers(n, d, K, variant, after):
-    m, a, c, x0 = _case(n, d, n)
+    m, a, c, x0 = _case(n, d, n, torus=variant == B.DETAG_VARIANT_TORUS)
     eta = orc.spectrum(m.to_dense()).eta
     p = oracle_problem(m, K, eta, 0.05, a, c, 0.1, 7)
     ref = orc.run(p, x0, 2)

@@ -51,12 +51,14 @@ def _guarded_state(torch, m, d, ld, K, eta, observe, variant, where):
     (5, 30, 48, 2, B.DETAG_VARIANT_DENSE), (32, 131, 132, 3, B.DETAG_VARIANT_DENSE), (3, 2, 4, 1, B.DETAG_VARIANT_DENSE),
     (33, 67, 68, 2, B.DETAG_VARIANT_DENSE), (50, 130, 136, 3, B.DETAG_VARIANT_DENSE), (64, 65, 68, 2, B.DETAG_VARIANT_DENSE),
     (64, 67, 72, 4, B.DETAG_VARIANT_RING), (96, 130, 132, 2, B.DETAG_VARIANT_RING),
+    (64, 67, 72, 4, B.DETAG_VARIANT_TORUS), (32, 130, 132, 2, B.DETAG_VARIANT_TORUS), (64, 3, 4, 2, B.DETAG_VARIANT_TORUS),
     (9, 77, 80, 3, B.DETAG_VARIANT_CSR), (70, 33, 36, 2, B.DETAG_VARIANT_CSR)])
 def test_nothing_outside_the_arrays_is_written(n, d, ld, K, variant):
     import torch
 
     rng = np.random.default_rng(n * 7 + d)
-    m = inputs.metropolis_weights(inputs.ring_graph(n))
+    graph = inputs.torus_graph(n // 8, 8) if variant == B.DETAG_VARIANT_TORUS else inputs.ring_graph(n)
+    m = inputs.metropolis_weights(graph)
     eta = orc.spectrum(m.to_dense()).eta
     for where in (B.DETAG_GRADIENT_AT_NEW_MODEL, B.DETAG_GRADIENT_AT_PHASE_START):
         for observe in (False, True):

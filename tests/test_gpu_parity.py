@@ -27,7 +27,7 @@ def _variants_for(m, K):
     out = [B.DETAG_VARIANT_CSR]
     st = B.detag_create(m.n, 8, m.row_ptr, m.col_idx, m.vals, K, 0.1, 0.1)
     try:
-        for v in (B.DETAG_VARIANT_DENSE, B.DETAG_VARIANT_RING):
+        for v in (B.DETAG_VARIANT_DENSE, B.DETAG_VARIANT_RING, B.DETAG_VARIANT_TORUS):
             try:
                 B.detag_set_variant(st, v)
                 out.append(v)
@@ -234,6 +234,52 @@ def test_circulant_band_variant(n, d, K, kind):
     x0 = rng.standard_normal((n, d)).astype(np.float32)
     _check_one_step(m, K, 0.3, 0.02, a, c, x0, 0.1, 5, variants=[B.DETAG_VARIANT_RING])
     _check_trajectory(m, K, 0.3, 0.02, a, c, x0, 0.1, 5, steps=5, variants=[B.DETAG_VARIANT_RING])
+
+
+def _block_circulant(kind, R):
+    """n = 8 R workers in R blocks of 8, block (r, r') a function of |r - r'| on the block cycle only."""
+    if kind == "torus":
+        return inputs.metropolis_weights(inputs.torus_graph(R, 8))
+    n = 8 * R
+    dense = np.zeros((n, n))
+    shift = np.roll(np.eye(R), 1, axis=1)
+    if kind == "anisotropic":  # different weights along the two axes of the torus
+        ring8 = np.roll(np.eye(8), 1, axis=1)
+        dense = 0.3 * np.eye(n) + 0.25 * np.kron(shift + shift.T, np.eye(8)) + 0.1 * np.kron(np.eye(R), ring8 + ring8.T)
+    else:  # "path_blocks": the blocks are NOT circulant (a path inside each block), only the block cycle is
+        inner = inputs.metropolis_weights(inputs.path_graph(8)).to_dense()
+        dense = 0.6 * np.kron(np.eye(R), inner) + 0.2 * np.kron(shift + shift.T, np.eye(8))
+    return inputs.csr_from_dense(dense)
+
+
+@pytest.mark.parametrize("R,d,K,kind", [(8, 130, 8, "torus"), (4, 67, 3, "torus"), (8, 1, 2, "torus"), (8, 1025, 4, "anisotropic"),
+                                         (4, 300, 5, "anisotropic"), (8, 259, 3, "path_blocks"), (4, 64, 6, "path_blocks")])
+def test_block_circulant_transform_variant(R, d, K, kind):
+    """Tori (uniform and anisotropic weights) and a block-circulant matrix whose blocks are not circulant: the
+    transform kernel must give the oracle's rounds, per element and over a trajectory, at ragged sizes."""
+    rng = np.random.default_rng(R * 100 + d)
+    m = _block_circulant(kind, R)
+    n = 8 * R
+    assert B.DETAG_VARIANT_TORUS in _variants_for(m, K)
+    eta = orc.spectrum(m.to_dense()).eta
+    a, c = _random_objective(rng, n, d, scale=0.2)
+    x0 = rng.standard_normal((n, d)).astype(np.float32)
+    _check_one_step(m, K, eta, 0.02, a, c, x0, 0.1, 5, j0=(1 << 32) + 7, variants=[B.DETAG_VARIANT_TORUS])
+    _check_trajectory(m, K, eta, 0.02, a, c, x0, 0.1, 5, steps=6, variants=[B.DETAG_VARIANT_TORUS])
+
+
+def test_transform_variant_is_refused_without_the_structure():
+    for m in (inputs.metropolis_weights(inputs.ring_graph(64)),              # circulant, but blocks at +1 and -1 differ
+              inputs.metropolis_weights(inputs.random_regular4_graph(32, 1)),
+              inputs.metropolis_weights(inputs.torus_graph(8, 4)),            # blocks of 8 straddle two rows of 4
+              inputs.metropolis_weights(inputs.torus_graph(3, 8))):           # n = 24
+        assert B.DETAG_VARIANT_TORUS not in _variants_for(m, 3)
+    cfg3 = inputs.gossip_matrix(inputs.CONFIGS["cfg3"])
+    st = B.detag_create(64, 128, cfg3.row_ptr, cfg3.col_idx, cfg3.vals, 8, 0.3, 0.01)
+    try:
+        assert B.detag_get_variant(st) == B.DETAG_VARIANT_TORUS  # what AUTO picks for the 8 x 8 torus
+    finally:
+        B.detag_destroy(st)
 
 
 def test_misuse_is_reported_not_faulted():

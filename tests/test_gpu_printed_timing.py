@@ -91,8 +91,8 @@ def test_torus_64_dense_polynomial_kernel():
     eta = orc.spectrum(m.to_dense()).eta
     a, c = _objective(rng, 64, 333, scale=0.2)
     x0 = rng.standard_normal((64, 333)).astype(np.float32)
-    _check_one_phase(m, 8, eta, 0.005, a, c, x0, 0.05, 2, [B.DETAG_VARIANT_DENSE, B.DETAG_VARIANT_CSR])
-    _check_trajectory(m, 8, eta, 0.005, a, c, x0, 0.05, 2, 5, [B.DETAG_VARIANT_DENSE])
+    _check_one_phase(m, 8, eta, 0.005, a, c, x0, 0.05, 2, [B.DETAG_VARIANT_DENSE, B.DETAG_VARIANT_CSR, B.DETAG_VARIANT_TORUS])
+    _check_trajectory(m, 8, eta, 0.005, a, c, x0, 0.05, 2, 5, [B.DETAG_VARIANT_DENSE, B.DETAG_VARIANT_TORUS])
 
 
 @pytest.mark.parametrize("n,d,K", [(64, 130, 16), (256, 129, 8)])
