@@ -178,13 +178,18 @@ void analyse_torus(detag_state* s) {
         }
   if (!(worst <= 1e-13 * std::fmax(1.0, scale))) return;
   s->torus = true;
-  // fragment order of the kernel: entry (p, k-step s, lane) is Phat_p[lane / 4][2 (lane % 4) + s]
+  // fragment order of the kernel: entry (p, k-step s, lane) is Phat_p[c'][c] with the contraction index
+  // c = lane % 4 + 4 s and the output position c' = pi(lane / 4), pi(2 q + e) = q + 4 e (see step_torus.cu)
   s->torus_frag.resize(static_cast<size_t>(R) * 2 * 32);
-  for (int p = 0; p < R; ++p)
+  // For R = 8 the kernel's butterflies leave out the basis' normalisation (1/sqrt(8) for the constant and the
+  // alternating vector, 1/2 for the others) on the way in and on the way out: both factors go into the block.
+  for (int p = 0; p < R; ++p) {
+    const double scale = R == 8 ? ((p == 0 || p == R - 1) ? 0.125 : 0.25) : 1.0;
     for (int st = 0; st < 2; ++st)
       for (int lane = 0; lane < 32; ++lane)
         s->torus_frag[(static_cast<size_t>(p) * 2 + st) * 32 + lane] =
-            phat[(static_cast<size_t>(p) * C + lane / 4) * C + 2 * (lane % 4) + st];
+            scale * phat[(static_cast<size_t>(p) * C + ((lane / 4) >> 1) + 4 * ((lane / 4) & 1)) * C + (lane % 4) + 4 * st];
+  }
 }
 
 bool torus_ok(const detag_state* s) { return s->torus && s->d <= 0x7fffffffLL; }

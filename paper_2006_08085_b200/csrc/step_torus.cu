@@ -9,28 +9,32 @@
 //     P = sum_p (q_p q_p^T) (x) Phat_p ,      Phat_p = P_K(Mhat_p) ,  Mhat_p = sum_k cos(2 pi f_p k / R) G_k
 // (G_k the 8 x 8 block at distance k, f_p the frequency of basis vector q_p; all built by the host in float64
 // and checked there against the dense polynomial).  Applying P to a slab then costs, per worker-coordinate and
-// array, R multiply-adds for the forward transform, 8 for the block product and R for the way back: 24 for
-// R = 8 instead of the 64 of the dense 64 x 64 product.
+// array, a transform along r, 8 multiply-adds for the block product and the transform back: about 13 operations
+// for R = 8 (butterflies) instead of the 64 of the dense 64 x 64 product.
 //
 // Mapping onto the float64 tensor instruction (mma m8n8k4): the eight coordinates of a warp's tile are the M
-// index, the position c is the contraction index (two k-steps of four) and the output position c' the N index:
+// index, the position c is the contraction index (two k-steps of four, c = kq + 4 s) and the output position c'
+// the N index, with the N columns permuted (column 2 kq + e stands for c' = kq + 4 e):
 //     D[coord][c'] = sum_c Zhat_p[coord][c] Phat_p[c'][c] .
-// With the k-steps taking c = 2 (lane % 4) + s, the A fragment a lane supplies and the C fragment it receives are
-// the SAME worker positions: lane (coord = lane / 4, kq = lane % 4) owns workers 8 r + 2 kq + e (r = 0..R-1,
-// e = 0, 1) of one coordinate for input and output alike.  So the transforms along r run inside the lane over its
-// own registers (dense R x R with compile-time coefficients; a quarter of them are zero and cost nothing), the tail of the
-// step (model update, noise, gradient, tracker fold) is lane-local, and every lane writes its results over the
-// very elements it read: the output needs no tile of its own.
+// The A fragment a lane supplies and the C fragment it receives are then the SAME worker positions: lane
+// (coord = lane / 4, kq = lane % 4) owns workers 8 r + kq + 4 e (r = 0..R-1, e = 0, 1) of one coordinate for input
+// and output alike.  So the transforms along r run inside the lane over its own registers, the tail of the step
+// (model update, noise, gradient, tracker fold) is lane-local, and every lane writes its results over the very
+// elements it read: the output needs no tile of its own.
 //
-// Shared memory holds tiles of [64 or 32 workers][64 coordinates] as two 32-coordinate halves in the 128-byte
-// swizzle of the tensor maps; with the ownership above every warp-wide access hits 32 different banks, and the
-// TMA stores undo the swizzle on the way out.  Roles of the persistent CTA (one per SM):
-//   producer  one thread: per slab two loads each of x, y into one of two short-lived stages (handed back as soon as
-//             the tracker contraction has read its operands) and of g, a, c into one of three long-lived stages
-//             (read in the tail, then overwritten with g', x', y');
+// Shared memory holds tiles of [64 or 32 workers][64 coordinates], loaded by ONE three-dimensional TMA box per
+// array and slab - {32 coordinates, 2 halves, all rows}, 128-byte swizzle - so that every row is fetched as one
+// contiguous 256-byte piece (boxes of 32 coordinates fetched on their own reach 0.71 of the HBM copy rate with
+// this access pattern, 256-byte pieces 0.88).  With the ownership above every warp-wide access hits 32 different
+// banks, and the TMA stores undo the swizzle on the way out.  The box walks whole 32-coordinate halves: the last
+// d % 32 columns of the arrays are patched into the stage, and written back, by the lanes that own them.
+// Roles of the persistent CTA (one per SM):
+//   loaders   two threads: per slab one box each of x, y into one of two short-lived stages (handed back as soon as
+//             the tracker contraction has read its operands), and one box each of g, a, c into one of three
+//             long-lived stages (read in the tail, then overwritten with g', x', y');
 //   consumers 16 warps in two groups taking alternate slabs; a warp owns 8 coordinates x all workers;
-//   storer    one thread: when a group's 8 warps have written their results, six TMA stores send the stage's three
-//             tiles out; once they have been read the stage goes back to the producer.
+//   storer    one thread: when a group's 8 warps have written their results, three TMA stores send the stage's
+//             tiles out; once they have been read the stage goes back to its loader.
 // Arithmetic: float64 on chip, every stored value rounded once; x' = P (x - alpha y) by linearity of AG_K, the
 // tracker fold as (y~ - g) + fl32(g') like the other kernels.  Every wait is bounded.
 #include <cuda.h>
@@ -48,17 +52,17 @@ namespace {
 
 constexpr int kC = 8;                  // workers per block = MMA contraction and N extent
 constexpr int kTS = 64;                // coordinates per slab
-constexpr int kHalfCols = 32;          // coordinates per swizzled half tile (128 bytes)
+constexpr int kHalfCols = 32;          // coordinates per 128-byte swizzle row
 constexpr int kXYStages = 2, kEStages = 3;
 constexpr int kTGroups = 2, kTGroupWarps = kTS / 8;
 constexpr int kTConsumerWarps = kTGroups * kTGroupWarps;
-constexpr int kTProducerWarp = kTConsumerWarps, kTStoreWarp = kTConsumerWarps + 1;
-constexpr int kTThreads = (kTConsumerWarps + 2) * 32;
+constexpr int kTLoadXYWarp = kTConsumerWarps, kTStoreWarp = kTConsumerWarps + 1, kTLoadEWarp = kTConsumerWarps + 2;
+constexpr int kTThreads = (kTConsumerWarps + 3) * 32;
 
 template <int R>
 struct TorusPlan {
   static constexpr int kRows = R * kC;
-  static constexpr int kTileFloats = kRows * kTS;          // one array of one slab: two halves of [rows][32]
+  static constexpr int kTileFloats = kRows * kTS;          // one array of one slab: [row][half][32]
   static constexpr int kTileBytes = kTileFloats * 4;
   static constexpr int kXYBytes = 2 * kTileBytes, kEBytes = 3 * kTileBytes;
   static constexpr int kFragDoubles = R * 2 * 32;          // Phat in fragment order: [p][k-step][lane]
@@ -70,62 +74,164 @@ struct TorusPlan {
 };
 
 struct TorusMaps {
-  CUtensorMap x, y, g, a, c;  // loads: boxes of [rows][32 coordinates], 128-byte swizzle, zero fill
-  CUtensorMap xs, ys, gs;     // stores: the same boxes over the columns below d & ~3
+  CUtensorMap x, y, g, a, c;  // loads: boxes {32 coordinates, 2 halves, all rows}, 128-byte swizzle, zero fill
+  CUtensorMap xs, ys, gs;     // stores: the same boxes
 };
 static_assert(sizeof(TorusMaps) <= sizeof(TensorMapSet), "tensor map storage");
 
-// [rows][32-coordinate box] tensor map with the 128-byte swizzle.
-inline bool make_swizzled_map(CUtensorMap* m, const float* base, int n, long long d, long long ld, int box_rows) {
+// View of an [n][ld] array as {32 coordinates, d / 32 halves at a stride of 128 bytes, n rows}: a box of two halves
+// is a slab of 64 coordinates whose rows are contiguous 256-byte pieces.  Only whole halves are in the view.
+inline bool make_half_map(CUtensorMap* m, const float* base, int n, long long d, long long ld) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
-  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(n)};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * sizeof(float)};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kHalfCols), static_cast<cuuint32_t>(box_rows)};
-  const cuuint32_t elem[2] = {1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, elem,
+  const long long halves = d / kHalfCols;
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(kHalfCols), static_cast<cuuint64_t>(halves > 0 ? halves : 1),
+                              static_cast<cuuint64_t>(n)};
+  const cuuint64_t strides[2] = {kHalfCols * sizeof(float), static_cast<cuuint64_t>(ld) * sizeof(float)};
+  const cuuint32_t box[3] = {static_cast<cuuint32_t>(kHalfCols), 2, static_cast<cuuint32_t>(n)};
+  const cuuint32_t elem[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, elem,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Gradient phase of a lane: g' = a (x_at - c) + sigma xi for its 2R elements, written over c in the stage (c is not
-// needed again; the tracker phase picks g' up from there).  x_at: the model at which the gradient is taken.
-// Noise: the Philox call of (coordinate, workers 8 r + 4 (kq / 2) .. + 3) serves this lane and its neighbour
-// kq ^ 1; each draws the calls of every other block r and they swap the word pairs they do not need themselves.
+__device__ __forceinline__ void slab_load(float* dst, const CUtensorMap* map, int half, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+          s_addr(dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(half), "r"(0), "r"(s_addr(bar))
+      : "memory");
+}
+
+__device__ __forceinline__ void slab_store(const CUtensorMap* map, int half, const float* src) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
+                   reinterpret_cast<uint64_t>(map)),
+               "r"(0), "r"(half), "r"(0), "r"(s_addr(src))
+               : "memory");
+}
+
+// 4 x 4 transpose over the four lanes that share a coordinate (lane bits 0 and 1): lane kq gives row kq = v[0..3]
+// and receives column kq.
+__device__ __forceinline__ void transpose_quad(float (&v)[4], int kq) {
+  const bool b0 = (kq & 1) != 0, b1 = (kq & 2) != 0;
+  float s0 = b0 ? v[0] : v[1], s1 = b0 ? v[2] : v[3];
+  float r0 = __shfl_xor_sync(0xffffffffu, s0, 1), r1 = __shfl_xor_sync(0xffffffffu, s1, 1);
+  if (b0) { v[0] = r0; v[2] = r1; } else { v[1] = r0; v[3] = r1; }
+  s0 = b1 ? v[0] : v[2];
+  s1 = b1 ? v[1] : v[3];
+  r0 = __shfl_xor_sync(0xffffffffu, s0, 2);
+  r1 = __shfl_xor_sync(0xffffffffu, s1, 2);
+  if (b1) { v[0] = r0; v[1] = r1; } else { v[2] = r0; v[3] = r1; }
+}
+
+// Transform of one worker column (this lane's R values along the block axis) into the Fourier components of the
+// block cycle, and back.  R = 8: butterflies of the real 8-point transform WITHOUT normalisation (20 operations
+// instead of 48; the host folds the two missing factors 1/8 resp. 1/4 into the per-frequency blocks).  Other R:
+// dense product with the orthonormal basis.  Component order as in torus_basis.h.
 template <int R>
-__device__ __forceinline__ void torus_gradient(const StepParams& p, const float* sa, float* sc, const int (&off_e)[2],
+__device__ __forceinline__ void torus_forward(const double (&z)[R], double (&w)[R]) {
+  if (R == 8) {
+    constexpr double c = 0.70710678118654752440;
+    const double s0 = z[0] + z[4], d0 = z[0] - z[4], s1 = z[1] + z[5], d1 = z[1] - z[5];
+    const double s2 = z[2] + z[6], d2 = z[2] - z[6], s3 = z[3] + z[7], d3 = z[3] - z[7];
+    const double t0 = s0 + s2, t1 = s1 + s3, u = d1 - d3, v = d1 + d3;
+    w[0] = t0 + t1;            // frequency 0
+    w[R - 1] = t0 - t1;        // frequency 4
+    w[1] = fma(c, u, d0);      // frequency 1: cosine, sine
+    w[2] = fma(c, v, d2);
+    w[3] = s0 - s2;            // frequency 2
+    w[4] = s1 - s3;
+    w[R - 3] = fma(-c, u, d0); // frequency 3
+    w[R - 2] = fma(c, v, -d2);
+  } else {
+#pragma unroll
+    for (int pf = 0; pf < R; ++pf) {
+      double acc = 0.0;
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+        if (torus_q(R, pf, r) != 0.0) acc = fma(torus_q(R, pf, r), z[r], acc);
+      w[pf] = acc;
+    }
+  }
+}
+
+template <int R>
+__device__ __forceinline__ void torus_backward(const double (&w)[R], double (&z)[R]) {
+  if (R == 8) {
+    constexpr double c = 0.70710678118654752440;
+    const double e0 = w[0] + w[R - 1], e1 = w[0] - w[R - 1];
+    const double p1 = w[1] + w[R - 3], p2 = w[2] - w[R - 2];  // C1 + C3, S1 - S3
+    const double q1 = w[1] - w[R - 3], q2 = w[2] + w[R - 2];  // C1 - C3, S1 + S3
+    const double a0 = e0 + w[3], a1 = e0 - w[3], b0 = e1 + w[4], b1 = e1 - w[4];
+    const double m0 = q1 + q2, m1 = q2 - q1;
+    z[0] = a0 + p1;
+    z[4] = a0 - p1;
+    z[2] = a1 + p2;
+    z[R - 2] = a1 - p2;
+    z[1] = fma(c, m0, b0);
+    z[R - 3] = fma(-c, m0, b0);
+    z[3] = fma(c, m1, b1);
+    z[R - 1] = fma(-c, m1, b1);
+  } else {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      double acc = 0.0;
+#pragma unroll
+      for (int pf = 0; pf < R; ++pf)
+        if (torus_q(R, pf, r) != 0.0) acc = fma(torus_q(R, pf, r), w[pf], acc);
+      z[r] = acc;
+    }
+  }
+}
+
+// P applied to this lane's two worker columns: forward transform of each (column(s, z) supplies column c = 2 kq + s),
+// one float64 MMA pair per frequency (contraction over the position inside the block, all four lanes of a coordinate
+// together) - torus_contract - then the transform back of the columns c' = 2 kq + e - torus_finish.
+template <int R, typename Column>
+__device__ __forceinline__ void torus_contract(double (&acc)[R][2], const double* frag, int lane, Column column) {
+#pragma unroll
+  for (int pf = 0; pf < R; ++pf) acc[pf][0] = acc[pf][1] = 0.0;
+#pragma unroll
+  for (int s = 0; s < 2; ++s) {
+    double z[R], w[R];
+    asm volatile("" ::: "memory");  // keeps the second column's loads behind the first column's arithmetic (registers)
+    column(s, z);
+    torus_forward<R>(z, w);
+#pragma unroll
+    for (int pf = 0; pf < R; ++pf) dmma(acc[pf], w[pf], frag[(pf * 2 + s) * 32 + lane]);
+  }
+}
+
+template <int R>
+__device__ __forceinline__ void torus_finish(const double (&acc)[R][2], int e, double (&out)[R]) {
+  double w[R];
+#pragma unroll
+  for (int pf = 0; pf < R; ++pf) w[pf] = acc[pf][e];
+  torus_backward<R>(w, out);
+}
+
+
+// Gradient phase of a lane: g' = a (x_at - c) + sigma xi for its 2R elements (element (r, e) at off + r * 512 + e * 256),
+// written over c in the stage (c is not needed again; the tracker phase picks g' up from there).  x_at: the model
+// at which the gradient is taken.  Noise: the lane's workers 8 r + 4 e + kq are position kq of the Philox quads
+// 2 r + e, which the four lanes of a coordinate share: each draws every fourth quad (all four normals of it) and a
+// 4 x 4 transpose over the lanes hands everybody its own position.
+template <int R>
+__device__ __forceinline__ void torus_gradient(const StepParams& p, const float* sa, float* sc, int off,
                                                const float (&x_at)[2][R], int kq, long long j, float sigma, bool noisy) {
   unsigned long long jn = static_cast<unsigned long long>(p.coord_offset + j);
-  // Ties the counter to the model values so that the compiler cannot start the generator's integer work while the
-  // contraction before this phase still holds its accumulators (it would spill them).
-  asm volatile("" : "+l"(jn) : "f"(x_at[0][0]), "f"(x_at[1][R - 1]));
-  const bool odd = (kq & 1) != 0;
 #pragma unroll
-  for (int h = 0; h < R / 2; ++h) {
-    float xi[2][2] = {{0.f, 0.f}, {0.f, 0.f}};  // [e][block 2h, 2h + 1]
+  for (int t = 0; t < R / 2; ++t) {  // quads 4 t .. 4 t + 3: blocks r = 2 t, 2 t + 1
+    float xi[4] = {0.f, 0.f, 0.f, 0.f};
     if (noisy) {
-      const int r_mine = 2 * h + (odd ? 1 : 0);
-      const Philox4 w = philox4x32_10(static_cast<uint32_t>(jn), static_cast<uint32_t>(jn >> 32),
-                                      static_cast<uint32_t>(2 * r_mine + (kq >> 1)), p.t_noise, p.seed_lo, p.seed_hi);
-      // even kq owns the first pair of words (workers +0, +1 of the quad), odd kq the second (workers +2, +3)
-      const uint32_t keep0 = odd ? w.r2 : w.r0, keep1 = odd ? w.r3 : w.r1;
-      const uint32_t give0 = odd ? w.r0 : w.r2, give1 = odd ? w.r1 : w.r3;
-      const uint32_t got0 = __shfl_xor_sync(0xffffffffu, give0, 1), got1 = __shfl_xor_sync(0xffffffffu, give1, 1);
-      float n0, n1, m0, m1;
-      box_muller(keep0, keep1, n0, n1);  // block r_mine
-      box_muller(got0, got1, m0, m1);    // the neighbour's block
-      xi[0][0] = odd ? m0 : n0;
-      xi[1][0] = odd ? m1 : n1;
-      xi[0][1] = odd ? n0 : m0;
-      xi[1][1] = odd ? n1 : m1;
+      normal_quad(p.seed_lo, p.seed_hi, jn, static_cast<uint32_t>(4 * t + kq), p.t_noise, xi);
+      transpose_quad(xi, kq);  // xi[i]: this lane's position of quad 4 t + i, i.e. r = 2 t + (i >> 1), e = i & 1
     }
 #pragma unroll
-    for (int b = 0; b < 2; ++b)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int r = 2 * h + b, o = off_e[e] + r * 256;
-        sc[o] = fmaf(sa[o], x_at[e][r] - sc[o], sigma * xi[e][b]);
-      }
+    for (int i = 0; i < 4; ++i) {
+      const int r = 2 * t + (i >> 1), e = i & 1, o = off + r * 512 + e * 256;
+      sc[o] = fmaf(sa[o], x_at[e][r] - sc[o], sigma * xi[i]);
+    }
   }
 }
 
@@ -167,46 +273,68 @@ step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, co
   // this CTA takes slabs blockIdx.x, blockIdx.x + gridDim.x, ...; k counts them
   const long long my_slabs = blockIdx.x < p.num_slabs ? (p.num_slabs - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
   const unsigned limit = p.spin_limit;
+  const long long d32 = p.d & ~31LL;  // columns below this travel by TMA, the rest by the lanes that own them
+  const int halves = static_cast<int>(d32 / kHalfCols);
 
-  if (warp == kTProducerWarp) {
+  if (warp == kTLoadXYWarp) {
+    // ---------------------------------------------------------------- x, y loader: runs ahead of the other one
     if (lane == 0) {
       long long k = 0;
       bool ok = true;
       for (; k < my_slabs; ++k) {
         if (p.stall_after >= 0 && k >= p.stall_after) return;  // self test: the loads stop, every waiter times out
-        const int sx = static_cast<int>(k % kXYStages), se = static_cast<int>(k % kEStages);
-        if (k >= kEStages) ok = bar_wait(&e_empty[se], ((k / kEStages) - 1) & 1, limit);
-        if (ok && k >= kXYStages) ok = bar_wait(&xy_empty[sx], ((k / kXYStages) - 1) & 1, limit);
+        const int sx = static_cast<int>(k % kXYStages);
+        if (k >= kXYStages) ok = bar_wait(&xy_empty[sx], ((k / kXYStages) - 1) & 1, limit);
         if (!ok) break;
-        const int col = static_cast<int>((blockIdx.x + k * gridDim.x) * kTS);
+        const int half = static_cast<int>((blockIdx.x + k * gridDim.x) * 2);
         float* tx = xy_mem + static_cast<size_t>(sx) * 2 * Plan::kTileFloats;
-        float* te = e_mem + static_cast<size_t>(se) * 3 * Plan::kTileFloats;
-        bar_expect_tx(&xy_full[sx], Plan::kXYBytes);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          tile_load(tx + h * (Plan::kTileFloats / 2), &maps.x, col + h * kHalfCols, 0, &xy_full[sx]);
-          tile_load(tx + Plan::kTileFloats + h * (Plan::kTileFloats / 2), &maps.y, col + h * kHalfCols, 0, &xy_full[sx]);
-        }
-        bar_expect_tx(&e_full[se], Plan::kEBytes);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          tile_load(te + h * (Plan::kTileFloats / 2), &maps.g, col + h * kHalfCols, 0, &e_full[se]);
-          tile_load(te + Plan::kTileFloats + h * (Plan::kTileFloats / 2), &maps.a, col + h * kHalfCols, 0, &e_full[se]);
-          tile_load(te + 2 * Plan::kTileFloats + h * (Plan::kTileFloats / 2), &maps.c, col + h * kHalfCols, 0, &e_full[se]);
+        const bool any = half < halves;  // a slab without a whole half is served entirely by its lanes
+        bar_expect_tx(&xy_full[sx], any ? Plan::kXYBytes : 0u);
+        if (any) {
+          slab_load(tx, &maps.x, half, &xy_full[sx]);
+          slab_load(tx + Plan::kTileFloats, &maps.y, half, &xy_full[sx]);
         }
       }
       if (!ok) {
         atomicExch(p.status, 1);
-        for (long long back = 1; back <= kEStages && back <= k; ++back) {  // drain copies still in flight (bounded)
+        for (long long back = 1; back <= kXYStages && back <= k; ++back) {  // drain copies still in flight (bounded)
           const long long q = k - back;
-          bar_wait(&e_full[q % kEStages], (q / kEStages) & 1, limit);
-          if (back <= kXYStages) bar_wait(&xy_full[q % kXYStages], (q / kXYStages) & 1, limit);
+          bar_wait(&xy_full[q % kXYStages], (q / kXYStages) & 1, limit);
         }
       }
     }
     return;
   }
-
+  if (warp == kTLoadEWarp) {
+    // ---------------------------------------------------------------- g, a, c loader
+    if (lane == 0) {
+      long long k = 0;
+      bool ok = true;
+      for (; k < my_slabs; ++k) {
+        if (p.stall_after >= 0 && k >= p.stall_after) return;
+        const int se = static_cast<int>(k % kEStages);
+        if (k >= kEStages) ok = bar_wait(&e_empty[se], ((k / kEStages) - 1) & 1, limit);
+        if (!ok) break;
+        const int half = static_cast<int>((blockIdx.x + k * gridDim.x) * 2);
+        float* te = e_mem + static_cast<size_t>(se) * 3 * Plan::kTileFloats;
+        const bool any = half < halves;
+        bar_expect_tx(&e_full[se], any ? Plan::kEBytes : 0u);
+        if (any) {
+          slab_load(te, &maps.g, half, &e_full[se]);
+          slab_load(te + Plan::kTileFloats, &maps.a, half, &e_full[se]);
+          slab_load(te + 2 * Plan::kTileFloats, &maps.c, half, &e_full[se]);
+        }
+      }
+      if (!ok) {
+        atomicExch(p.status, 1);
+        for (long long back = 1; back <= kEStages && back <= k; ++back) {
+          const long long q = k - back;
+          bar_wait(&e_full[q % kEStages], (q / kEStages) & 1, limit);
+        }
+      }
+    }
+    return;
+  }
   if (warp == kTStoreWarp) {
     if (lane == 0) {
       for (long long k = 0; k < my_slabs; ++k) {
@@ -216,15 +344,11 @@ step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, co
           break;
         }
         const float* te = e_mem + static_cast<size_t>(se) * 3 * Plan::kTileFloats;  // now [g' | x' | y']
-        const int col = static_cast<int>((blockIdx.x + k * gridDim.x) * kTS);
-        const long long d_tma = p.d & ~3LL;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          if (col + h * kHalfCols < d_tma) {
-            tile_store(&maps.gs, col + h * kHalfCols, 0, te + h * (Plan::kTileFloats / 2));
-            tile_store(&maps.xs, col + h * kHalfCols, 0, te + Plan::kTileFloats + h * (Plan::kTileFloats / 2));
-            tile_store(&maps.ys, col + h * kHalfCols, 0, te + 2 * Plan::kTileFloats + h * (Plan::kTileFloats / 2));
-          }
+        const int half = static_cast<int>((blockIdx.x + k * gridDim.x) * 2);
+        if (half < halves) {  // the stores clip at the last whole half
+          slab_store(&maps.gs, half, te);
+          slab_store(&maps.xs, half, te + Plan::kTileFloats);
+          slab_store(&maps.ys, half, te + 2 * Plan::kTileFloats);
         }
         store_commit();
         store_wait_read();  // the stage may be refilled now
@@ -241,26 +365,71 @@ step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, co
   const double alpha = p.alpha;
   const float sigma = static_cast<float>(p.sigma);
   const bool noisy = p.sigma != 0.0;
-  const long long d_tma = p.d & ~3LL;
-  // Float offset of this lane's element (r = 0, e) inside an array's tile; element (r, e) lies r * 256 further.
-  // Tile = [half][row][32]; 16-byte chunk index XOR (row & 7) is the tensor maps' 128-byte swizzle.
-  int off_e[2];
-#pragma unroll
-  for (int e = 0; e < 2; ++e) {
-    const int row7 = 2 * kq + e;  // (8 r + 2 kq + e) & 7
-    const int chunk = 2 * (tile & 3) + (crow >> 2);
-    off_e[e] = (tile >> 2) * (Plan::kTileFloats / 2) + row7 * kHalfCols + (((chunk ^ row7) << 2) | (crow & 3));
-  }
+  // Float offset of this lane's element (r = 0, e = 0) inside an array's tile; element (r, e) - worker
+  // 8 r + kq + 4 e - lies r * 512 + e * 256 further.  Tile = [row][half][32]; the 16-byte chunk index is XORed with
+  // the low three bits of the 128-byte row number 2 * row + half (the tensor maps' swizzle), which for this lane's
+  // rows is always 2 kq + half.
+  const int half_of_tile = tile >> 2;
+  const int chunk = 2 * (tile & 3) + (crow >> 2);
+  const int off = kq * kTS + half_of_tile * kHalfCols + (((chunk ^ ((2 * kq + half_of_tile) & 7)) << 2) | (crow & 3));
 
   for (long long k = group; k < my_slabs; k += kTGroups) {
     const int sx = static_cast<int>(k % kXYStages), se = static_cast<int>(k % kEStages);
     bool ok = true;
+    if (lane == 0) ok = bar_wait(&xy_full[sx], (k / kXYStages) & 1, limit);
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    if (!ok) {
+      if (lane == 0) atomicExch(p.status, 1);
+      return;
+    }
+    float* sxp = xy_mem + static_cast<size_t>(sx) * 2 * Plan::kTileFloats;
+    float* syp = sxp + Plan::kTileFloats;
+    float* sg = e_mem + static_cast<size_t>(se) * 3 * Plan::kTileFloats;
+    float* sa = sg + Plan::kTileFloats;
+    float* sc = sa + Plan::kTileFloats;
+    const long long slab = blockIdx.x + k * gridDim.x;
+    const long long j = slab * kTS + tile * 8 + crow;  // this lane's coordinate
+    const bool active = slab * kTS + tile * 8 < p.d;   // a tile wholly beyond column d computes nothing
+    const bool mine = j >= d32 && j < p.d;             // a column the TMA boxes do not reach: this lane moves it
+    if (mine) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e)
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const long long g_off = static_cast<long long>(8 * r + kq + 4 * e) * p.ld + j;
+          sxp[off + r * 512 + e * 256] = p.x[g_off];
+          syp[off + r * 512 + e * 256] = p.y[g_off];
+        }
+    }
+
+    // Registers are the scarce resource here (2R values per array and lane, float64 accumulators): the phases below
+    // run one after the other, read their operands from the stages when they need them and park what a later
+    // phase needs in the lane's own slots - g' over c, x' over a (both read just before), finally g' over g and y'
+    // over c.
+    float xv[2][R];  // x'
+    if (active) {
+      // ---- model: x' = P (x - alpha y), by linearity of AG_K
+      double acc[R][2];
+      torus_contract<R>(acc, frag, lane, [&](int s, double (&z)[R]) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const int o = off + r * 512 + s * 256;
+          z[r] = fma(-alpha, static_cast<double>(syp[o]), static_cast<double>(sxp[o]));
+        }
+      });
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        double out[R];
+        torus_finish<R>(acc, e, out);
+#pragma unroll
+        for (int r = 0; r < R; ++r) xv[e][r] = static_cast<float>(out[r]);  // rounded once
+      }
+    }
+    // g, a, c are needed from here on; their loads had the model contraction to arrive in
     if (lane == 0) {
-      ok = bar_wait(&xy_full[sx], (k / kXYStages) & 1, limit);
-      // The g, a, c stage last held slab k - 3, which belongs to the other group (odd stage count): a parity wait
-      // must not start before that phase has completed, or it could not tell the two apart.
-      if (ok && k >= kEStages)
-        ok = count_wait(&seen[(k - kEStages) % kTGroups], static_cast<unsigned>(k - kEStages + 1), limit);
+      // The stage last held slab k - 3, which belongs to the other group (odd stage count): a parity wait must not
+      // start before that phase has completed, or it could not tell the two apart.
+      if (k >= kEStages) ok = count_wait(&seen[(k - kEStages) % kTGroups], static_cast<unsigned>(k - kEStages + 1), limit);
       if (ok) ok = bar_wait(&e_full[se], (k / kEStages) & 1, limit);
       if (ok && tile == 0) count_publish(&seen[group], static_cast<unsigned>(k + 1));
     }
@@ -269,121 +438,72 @@ step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, co
       if (lane == 0) atomicExch(p.status, 1);
       return;
     }
-    const float* sxp = xy_mem + static_cast<size_t>(sx) * 2 * Plan::kTileFloats;
-    const float* syp = sxp + Plan::kTileFloats;
-    float* sg = e_mem + static_cast<size_t>(se) * 3 * Plan::kTileFloats;
-    float* sa = sg + Plan::kTileFloats;
-    float* sc = sa + Plan::kTileFloats;
-    const long long slab = blockIdx.x + k * gridDim.x;
-    const long long j = slab * kTS + tile * 8 + crow;  // this lane's coordinate
-    const bool active = slab * kTS + tile * 8 < p.d;   // a tile wholly beyond column d computes nothing
-
-    bool released = false;
-    if (active) {
-      // Registers are the scarce resource here (2R values per array and lane, float64 accumulators): the phases
-      // below run one after the other, read their operands from the stages when they need them and park what a
-      // later phase needs in the lane's own slots - x' over a, then g' over c (both read just before), finally g'
-      // over g and y' over c.
-      float xv[2][R];  // the model at which the gradient is taken, then x'
-      if (kAtStart) {  // Algorithm 2 as printed: the gradient at the model the step started from
-#pragma unroll
-        for (int e = 0; e < 2; ++e)
-#pragma unroll
-          for (int r = 0; r < R; ++r) xv[e][r] = sxp[off_e[e] + r * 256];
-        torus_gradient<R>(p, sa, sc, off_e, xv, kq, j, sigma, noisy);
-      }
-      // ---- model: x' = P (x - alpha y), by linearity of AG_K
-      {
-        double acc[R][2];
-#pragma unroll
-        for (int pf = 0; pf < R; ++pf) acc[pf][0] = acc[pf][1] = 0.0;
-#pragma unroll
-        for (int s = 0; s < 2; ++s) {  // k-step s: this lane's worker column c = 2 kq + s
-          double z[R];
-#pragma unroll
-          for (int r = 0; r < R; ++r) {
-            const int o = off_e[s] + r * 256;
-            z[r] = fma(-alpha, static_cast<double>(syp[o]), static_cast<double>(sxp[o]));
-          }
-#pragma unroll
-          for (int pf = 0; pf < R; ++pf) {
-            double zh = 0.0;  // forward transform: component pf of the column
-#pragma unroll
-            for (int r = 0; r < R; ++r) if (torus_q(R, pf, r) != 0.0) zh = fma(torus_q(R, pf, r), z[r], zh);
-            dmma(acc[pf], zh, frag[(pf * 2 + s) * 32 + lane]);
-          }
-        }
-#pragma unroll
-        for (int e = 0; e < 2; ++e)
-#pragma unroll
-          for (int r = 0; r < R; ++r) {
-            double v = 0.0;  // transform back: worker (r, 2 kq + e)
-#pragma unroll
-            for (int pf = 0; pf < R; ++pf) if (torus_q(R, pf, r) != 0.0) v = fma(torus_q(R, pf, r), acc[pf][e], v);
-            xv[e][r] = static_cast<float>(v);  // x', rounded once
-          }
-      }
-      if (!kAtStart) torus_gradient<R>(p, sa, sc, off_e, xv, kq, j, sigma, noisy);  // at the new model
+    if (mine) {
 #pragma unroll
       for (int e = 0; e < 2; ++e)
 #pragma unroll
-        for (int r = 0; r < R; ++r) sa[off_e[e] + r * 256] = xv[e][r];  // x' takes a's place
-      // ---- tracker: y~ = P y, then the fold (y~ - g) + g'
-      {
-        double acc[R][2];
-#pragma unroll
-        for (int pf = 0; pf < R; ++pf) acc[pf][0] = acc[pf][1] = 0.0;
-#pragma unroll
-        for (int s = 0; s < 2; ++s) {
-          double z[R];
-#pragma unroll
-          for (int r = 0; r < R; ++r) z[r] = static_cast<double>(syp[off_e[s] + r * 256]);
-          if (s == 1) {  // the last read of the x, y stage: it can be refilled
-            __syncwarp();
-            if (lane == 0) bar_arrive(&xy_empty[sx]);
-            released = true;
-          }
-#pragma unroll
-          for (int pf = 0; pf < R; ++pf) {
-            double zh = 0.0;
-#pragma unroll
-            for (int r = 0; r < R; ++r) if (torus_q(R, pf, r) != 0.0) zh = fma(torus_q(R, pf, r), z[r], zh);
-            dmma(acc[pf], zh, frag[(pf * 2 + s) * 32 + lane]);
-          }
+        for (int r = 0; r < R; ++r) {
+          const long long g_off = static_cast<long long>(8 * r + kq + 4 * e) * p.ld + j;
+          sg[off + r * 512 + e * 256] = p.g[g_off];
+          sa[off + r * 512 + e * 256] = p.a[g_off];
+          sc[off + r * 512 + e * 256] = p.c[g_off];
         }
-        const bool in_d = j < p.d;
+    }
+    if (active) {
+      if (kAtStart) {  // Algorithm 2 as printed: the gradient at the model the step started from (still staged)
+        float xold[2][R];
+#pragma unroll
+        for (int e = 0; e < 2; ++e)
+#pragma unroll
+          for (int r = 0; r < R; ++r) xold[e][r] = sxp[off + r * 512 + e * 256];
+        torus_gradient<R>(p, sa, sc, off, xold, kq, j, sigma, noisy);
+      } else {
+        torus_gradient<R>(p, sa, sc, off, xv, kq, j, sigma, noisy);
+      }
+#pragma unroll
+      for (int e = 0; e < 2; ++e)
+#pragma unroll
+        for (int r = 0; r < R; ++r) sa[off + r * 512 + e * 256] = xv[e][r];  // x' takes a's place
+    }
+    // ---- tracker: y~ = P y, then the fold (y~ - g) + g'
+    double acc[R][2];
+    if (active) {
+      torus_contract<R>(acc, frag, lane, [&](int s, double (&z)[R]) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) z[r] = static_cast<double>(syp[off + r * 512 + s * 256]);
+      });
+    }
+    if (mine) fence_async_shared();  // this lane wrote into the x, y stage: order that before the next load into it
+    __syncwarp();
+    if (lane == 0) bar_arrive(&xy_empty[sx]);  // that was the last read of the x, y stage: it can be refilled
+    if (active) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        double out[R];
+        torus_finish<R>(acc, e, out);
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const int o = off + r * 512 + e * 256;
+          const float go = sc[o];  // g', parked there by the gradient phase
+          const float yo = static_cast<float>((out[r] - static_cast<double>(sg[o])) + static_cast<double>(go));
+          sg[o] = go;
+          sc[o] = yo;
+          if (p.y_obs != nullptr && j < p.d)  // optional observer: the gossiped tracker, stored directly
+            p.y_obs[static_cast<long long>(8 * r + kq + 4 * e) * p.ld + j] = static_cast<float>(out[r]);
+        }
+      }
+      if (mine) {  // the last d % 32 columns go out directly
 #pragma unroll
         for (int e = 0; e < 2; ++e)
 #pragma unroll
           for (int r = 0; r < R; ++r) {
-            double v = 0.0;
-#pragma unroll
-            for (int pf = 0; pf < R; ++pf) if (torus_q(R, pf, r) != 0.0) v = fma(torus_q(R, pf, r), acc[pf][e], v);
-            const int o = off_e[e] + r * 256;
-            const float go = sc[o];  // g', parked there by the gradient phase
-            const float yo = static_cast<float>((v - static_cast<double>(sg[o])) + static_cast<double>(go));
-            sg[o] = go;
-            sc[o] = yo;
-            if (p.y_obs != nullptr && in_d)  // optional observer: the gossiped tracker, stored directly
-              p.y_obs[static_cast<long long>(8 * r + 2 * kq + e) * p.ld + j] = static_cast<float>(v);
+            const int o = off + r * 512 + e * 256;
+            const long long g_off = static_cast<long long>(8 * r + kq + 4 * e) * p.ld + j;
+            p.x[g_off] = sa[o];
+            p.y[g_off] = sc[o];
+            p.g[g_off] = sg[o];
           }
-        if (in_d && j >= d_tma) {  // TMA clips stores at 16-byte granularity: the last d % 4 columns go out directly
-#pragma unroll
-          for (int e = 0; e < 2; ++e)
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-              const int o = off_e[e] + r * 256;
-              const long long off = static_cast<long long>(8 * r + 2 * kq + e) * p.ld + j;
-              p.x[off] = sa[o];
-              p.y[off] = sc[o];
-              p.g[off] = sg[o];
-            }
-        }
       }
-    }
-    if (!released) {  // idle tile: same protocol, nothing computed
-      __syncwarp();
-      if (lane == 0) bar_arrive(&xy_empty[sx]);
     }
     fence_async_shared();  // results visible to the TMA stores
     __syncwarp();
@@ -399,16 +519,13 @@ bool torus_variant_available(int n) { return (n == 32 || n == 64) && encode_tile
 
 bool build_maps_torus(const StepParams& p, TensorMapSet* out) {
   TorusMaps& m = *reinterpret_cast<TorusMaps*>(out->bytes);
-  const long long d_tma = p.d & ~3LL;
-  if (!make_swizzled_map(&m.x, p.x, p.n, p.d, p.ld, p.n) || !make_swizzled_map(&m.y, p.y, p.n, p.d, p.ld, p.n) ||
-      !make_swizzled_map(&m.g, p.g, p.n, p.d, p.ld, p.n) || !make_swizzled_map(&m.a, p.a, p.n, p.d, p.ld, p.n) ||
-      !make_swizzled_map(&m.c, p.c, p.n, p.d, p.ld, p.n))
+  if (!make_half_map(&m.x, p.x, p.n, p.d, p.ld) || !make_half_map(&m.y, p.y, p.n, p.d, p.ld) ||
+      !make_half_map(&m.g, p.g, p.n, p.d, p.ld) || !make_half_map(&m.a, p.a, p.n, p.d, p.ld) ||
+      !make_half_map(&m.c, p.c, p.n, p.d, p.ld))
     return false;
-  if (d_tma > 0 && (!make_swizzled_map(&m.xs, p.x, p.n, d_tma, p.ld, p.n) ||
-                    !make_swizzled_map(&m.ys, p.y, p.n, d_tma, p.ld, p.n) ||
-                    !make_swizzled_map(&m.gs, p.g, p.n, d_tma, p.ld, p.n)))
-    return false;
-  if (d_tma == 0) m.xs = m.ys = m.gs = m.x;  // never used
+  m.xs = m.x;
+  m.ys = m.y;
+  m.gs = m.g;
   return true;
 }
 
