@@ -17,7 +17,7 @@ namespace {
 size_t align_up(size_t v) { return (v + detag::kWsAlign - 1) / detag::kWsAlign * detag::kWsAlign; }
 
 struct WsLayout {
-  size_t status, result, row_ptr, col_idx, vals, poly, torus, partials, total;
+  size_t status, result, row_ptr, col_idx, vals, poly, torus, circ_row, partials, total;
 };
 
 WsLayout ws_layout(const detag_state* s) {
@@ -36,6 +36,8 @@ WsLayout ws_layout(const detag_state* s) {
   off += align_up(s->poly.size() * sizeof(double));
   l.torus = off;
   off += align_up(s->torus_frag.size() * sizeof(double));
+  l.circ_row = off;
+  off += align_up(s->circ_row.size() * sizeof(double));
   l.partials = off;
   off += align_up(detag::kMaxPartials * sizeof(double));
   l.total = off;
@@ -110,6 +112,7 @@ void analyse_circulant(detag_state* s) {
       if (delta > hb) hb = delta;
     }
   s->half_band = hb;
+  if (n <= 256) s->circ_row = cur;  // p(0 .. n-1): the dense mode of the circulant kernel looks its fragments up here
   if (hb <= 16 && n >= 2 * hb + 1)
     for (int delta = -16; delta <= 16; ++delta)
       s->band[delta + 16] = (delta >= -hb && delta <= hb) ? cur[((delta % n) + n) % n] : 0.0;
@@ -194,8 +197,11 @@ void analyse_torus(detag_state* s) {
 
 bool torus_ok(const detag_state* s) { return s->torus && s->d <= 0x7fffffffLL; }
 
+// The circulant kernel: band mode while the polynomial's half-band is at most 16, dense mode (n <= 256) beyond.
+bool ring_band(const detag_state* s) { return detag::ring_variant_available(s->n, s->half_band); }
+
 bool band_ok(const detag_state* s) {
-  return s->circulant && s->d <= 0x7fffffffLL && detag::band_variant_available(s->n, s->half_band);
+  return s->circulant && s->d <= 0x7fffffffLL && (ring_band(s) || detag::ring_dense_available(s->n));
 }
 
 int step_mode(const detag_state* s) {
@@ -222,6 +228,7 @@ StepParams make_params(const detag_state* s) {
   p.vals = s->d_vals;
   p.poly = s->d_poly;
   p.torus = s->d_torus;
+  p.circ_row = s->d_circ_row;
   p.eta = s->eta;
   p.alpha = s->alpha;
   p.sigma = s->sigma;
@@ -249,13 +256,18 @@ bool dense_ok(const detag_state* s) {
 // and array instead of 64.
 bool variant_runs_mode(const detag_state* s, int variant) {
   if (step_mode(s) == detag::kModeDetag) return true;
+  if (variant == DETAG_VARIANT_RING) return step_mode(s) == detag::kModeDpsgd;
   return variant == DETAG_VARIANT_CSR || (variant == DETAG_VARIANT_DENSE && s->n <= 32);
 }
 
 int resolve_variant(const detag_state* s) {
   if (s->variant_forced != DETAG_VARIANT_AUTO) return s->variant_forced;
+  // a ring whose band fits takes the circulant kernel from n = 64 on; with a dense polynomial only beyond the
+  // reach of the 64-row dense kernel
+  const bool ring = band_ok(s) && (ring_band(s) || s->n > detag::kMaxDenseWorkers);
+  if (step_mode(s) == detag::kModeDpsgd && s->n > 32 && ring) return DETAG_VARIANT_RING;
   if (step_mode(s) != detag::kModeDetag) return (s->n <= 32 && dense_ok(s)) ? DETAG_VARIANT_DENSE : DETAG_VARIANT_CSR;
-  if (s->n > 32 && band_ok(s)) return DETAG_VARIANT_RING;
+  if (s->n > 32 && ring) return DETAG_VARIANT_RING;
   if (s->n > 32 && torus_ok(s)) return DETAG_VARIANT_TORUS;
   if (dense_ok(s)) return DETAG_VARIANT_DENSE;
   return DETAG_VARIANT_CSR;
@@ -274,7 +286,7 @@ int query_device(detag_state* s) {
 }
 
 // Kernel families that take tensor maps.
-enum { kFamilyMma = 1, kFamilyBand = 2, kFamilyTorus = 3 };
+enum { kFamilyMma = 1, kFamilyBand = 2, kFamilyTorus = 3, kFamilyRing = 4 };
 
 // Tensor maps for the buffers in `p`: built on first use, then found again by buffer addresses and sizes
 // (detag_step always hits; detag_step_host cycles through its two chunk slots and the ragged last chunk).
@@ -299,6 +311,7 @@ const detag::TensorMapSet* maps_for(detag_state* s, int family, const StepParams
   en.family = 0;  // invalid until built
   const bool ok = family == kFamilyMma    ? detag::build_maps_mma(p, &en.maps)
                   : family == kFamilyBand ? detag::build_maps_band(p, &en.maps)
+                  : family == kFamilyRing ? detag::build_maps_ring(p, &en.maps)
                                           : detag::build_maps_torus(p, &en.maps);
   if (!ok) return nullptr;
   en.family = family;
@@ -320,15 +333,39 @@ int launch_step(detag_state* s, StepParams& p, cudaStream_t stream) {
   if (p.mode == detag::kModeExternal && !p.g_ext)
     return fail(s, DETAG_ERR_UNBOUND, "caller-written gradients selected but no gradient array given");
   switch (variant) {
-    case DETAG_VARIANT_DENSE:
-    case DETAG_VARIANT_RING: {
-      const bool mma = variant == DETAG_VARIANT_DENSE && p.n <= 32;
+    case DETAG_VARIANT_DENSE: {
+      const bool mma = p.n <= 32;
       const detag::TensorMapSet* maps = maps_for(s, mma ? kFamilyMma : kFamilyBand, p);
       if (!maps) return fail(s, DETAG_ERR_CUDA, "tensor map encoding failed");
-      if (mma)
-        e = detag::launch_step_mma(p, *maps, s->sm_count, stream);
-      else
-        e = detag::launch_step_band(p, *maps, variant == DETAG_VARIANT_RING ? s->band : nullptr, s->sm_count, stream);
+      e = mma ? detag::launch_step_mma(p, *maps, s->sm_count, stream)
+              : detag::launch_step_band(p, *maps, nullptr, s->sm_count, stream);
+      break;
+    }
+    case DETAG_VARIANT_RING: {
+      // the circulant kernel takes whole 64-coordinate slabs; the last d % 64 columns go to the generic kernel
+      const long long d_main = p.d & ~63LL;
+      if (d_main > 0) {
+        StepParams pm = p;
+        pm.d = d_main;
+        const detag::TensorMapSet* maps = maps_for(s, kFamilyRing, pm);
+        if (!maps) return fail(s, DETAG_ERR_CUDA, "tensor map encoding failed");
+        e = detag::launch_step_ring(pm, *maps, ring_band(s) ? s->band : nullptr, p.circ_row, s->sm_count, stream);
+        if (e != 0) return fail_cuda(s, e, "step kernel launch");
+      }
+      if (d_main < p.d) {
+        StepParams pt = p;
+        pt.d = p.d - d_main;
+        pt.coord_offset = p.coord_offset + d_main;
+        pt.x = p.x + d_main;
+        pt.y = p.y + d_main;
+        pt.g = p.g + d_main;
+        pt.a = p.a + d_main;
+        pt.c = p.c + d_main;
+        if (p.y_obs) pt.y_obs = p.y_obs + d_main;
+        const int rc = detag::plan_step_csr(pt, s->smem_optin);
+        if (rc != DETAG_OK) return fail(s, rc, "graph too large for the shared-memory plan");
+        e = detag::launch_step_csr(pt, s->sm_count, stream);
+      }
       break;
     }
     case DETAG_VARIANT_TORUS: {
@@ -430,6 +467,7 @@ int detag_bind(detag_state* s, int64_t ld, float* x, float* y, float* g, const f
   s->d_vals = reinterpret_cast<double*>(base + l.vals);
   s->d_poly = s->poly.empty() ? nullptr : reinterpret_cast<double*>(base + l.poly);
   s->d_torus = s->torus_frag.empty() ? nullptr : reinterpret_cast<double*>(base + l.torus);
+  s->d_circ_row = s->circ_row.empty() ? nullptr : reinterpret_cast<double*>(base + l.circ_row);
   s->d_partials = reinterpret_cast<double*>(base + l.partials);
 
   e = cudaMemset(base, 0, detag::kWsAlign);
@@ -443,6 +481,8 @@ int detag_bind(detag_state* s, int64_t ld, float* x, float* y, float* g, const f
     e = cudaMemcpy(s->d_poly, s->poly.data(), s->poly.size() * sizeof(double), cudaMemcpyHostToDevice);
   if (e == cudaSuccess && s->d_torus)
     e = cudaMemcpy(s->d_torus, s->torus_frag.data(), s->torus_frag.size() * sizeof(double), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess && s->d_circ_row)
+    e = cudaMemcpy(s->d_circ_row, s->circ_row.data(), s->circ_row.size() * sizeof(double), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) return fail_cuda(s, e, "detag_bind: workspace upload");
 
   s->ld = ld;
@@ -492,7 +532,7 @@ int detag_set_variant(detag_state* s, int variant) {
     case DETAG_VARIANT_RING:
       if (!band_ok(s))
         return fail(s, DETAG_ERR_UNSUPPORTED,
-                    "detag_set_variant: ring variant needs a circulant matrix, n a multiple of 32, n >= 64, K*bandwidth <= 16");
+                    "detag_set_variant: ring variant needs a circulant matrix, n a multiple of 32, n >= 64, and K*bandwidth <= 16 or n <= 256");
       break;
     default:
       return fail(s, DETAG_ERR_ARG, "detag_set_variant: unknown variant");
@@ -704,6 +744,9 @@ int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* 
   if (e == cudaSuccess && !s->torus_frag.empty())
     e = cudaMemcpyAsync(base + l.torus, s->torus_frag.data(), s->torus_frag.size() * sizeof(double),
                         cudaMemcpyHostToDevice, user);
+  if (e == cudaSuccess && !s->circ_row.empty())
+    e = cudaMemcpyAsync(base + l.circ_row, s->circ_row.data(), s->circ_row.size() * sizeof(double),
+                        cudaMemcpyHostToDevice, user);
   if (e == cudaSuccess) e = cudaEventRecord(s->host_event[2], user);
   for (int k = 0; k < 2 && e == cudaSuccess; ++k) e = cudaStreamWaitEvent(s->host_stream[k], s->host_event[2], 0);
   if (e != cudaSuccess) return fail_cuda(s, e, "detag_step_host: table upload");
@@ -714,6 +757,7 @@ int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* 
   p.vals = reinterpret_cast<double*>(base + l.vals);
   p.poly = s->poly.empty() ? nullptr : reinterpret_cast<double*>(base + l.poly);
   p.torus = s->torus_frag.empty() ? nullptr : reinterpret_cast<double*>(base + l.torus);
+  p.circ_row = s->circ_row.empty() ? nullptr : reinterpret_cast<double*>(base + l.circ_row);
   p.status = status_word;
   p.y_obs = nullptr;
   p.t_noise = static_cast<uint32_t>(s->t + 1);

@@ -39,6 +39,7 @@ struct StepParams {
   const int32_t* col_idx;
   const double* vals;
   const double* poly;  // dense P_K(M), row-major n x n (null when n > kMaxDenseWorkers)
+  const double* circ_row;  // circulant kernel, dense mode: the first row of P_K(M) (or null)
   const double* torus; // block-circulant kernel: per-frequency 8 x 8 polynomial blocks in fragment order (or null)
   double eta;
   double alpha;
@@ -87,6 +88,12 @@ bool dense_window_available(int n);                // the band kernel's dense mo
 bool build_maps_band(const StepParams& p, TensorMapSet* maps);
 int launch_step_band(StepParams p, const TensorMapSet& maps, const double* band /* null: dense mode */, int sm_count,
                      cudaStream_t stream);
+// circulant kernel (step_ring.cu): n % 32 == 0, 64 <= n <= 1024; band mode for half-band <= 16, dense mode for n <= 256
+bool ring_variant_available(int n, int half_band);
+bool ring_dense_available(int n);
+bool build_maps_ring(const StepParams& p, TensorMapSet* maps);  // p.d a multiple of 64
+int launch_step_ring(StepParams p, const TensorMapSet& maps, const double* band /* null: dense mode */,
+                     const double* p_row /* device: first row of P, dense mode */, int sm_count, cudaStream_t stream);
 bool torus_variant_available(int n);               // block-circulant kernel: n = 32 or 64 (4 or 8 blocks of 8)
 bool build_maps_torus(const StepParams& p, TensorMapSet* maps);
 int launch_step_torus(StepParams p, const TensorMapSet& maps, const double* phat_frag /* device */, int sm_count,
@@ -110,6 +117,7 @@ struct detag_state {
   bool circulant = false;    // every row of M is the previous one shifted by one
   int half_band = 0;         // of the circulant P_K(M): P[i][(i+delta) mod n] = 0 for |delta| > half_band
   double band[33] = {0};     // p(delta) at index delta + 16, valid when circulant and half_band <= 16
+  std::vector<double> circ_row;  // first row of the circulant P_K(M) (kept when n <= 256)
   // block-circulant structure with 8-worker blocks, symmetric in the block distance (tori): the per-frequency
   // 8 x 8 polynomial blocks in MMA fragment order
   bool torus = false;
@@ -137,6 +145,7 @@ struct detag_state {
   double* d_vals = nullptr;
   double* d_poly = nullptr;
   double* d_torus = nullptr;
+  double* d_circ_row = nullptr;
   double* d_partials = nullptr;
 
   double sigma = 0.0;

@@ -34,8 +34,11 @@ def _graph(kind, n):
     raise ValueError(kind)
 
 
-def _variants(n):
-    return [B.DETAG_VARIANT_CSR] + ([B.DETAG_VARIANT_DENSE] if n <= 32 else [])
+def _variants(n, dpsgd_ring=False):
+    out = [B.DETAG_VARIANT_CSR] + ([B.DETAG_VARIANT_DENSE] if n <= 32 else [])
+    if dpsgd_ring and n >= 64 and n % 32 == 0:
+        out.append(B.DETAG_VARIANT_RING)  # the circulant kernel also runs D-PSGD
+    return out
 
 
 # ----------------------------------------------------------------------------- caller-written gradients
@@ -136,7 +139,8 @@ def _objective(rng, n, d):
 @pytest.mark.parametrize("n,d,K,eta_mode,kind", [(8, 300, 1, "zero", "ring"), (16, 1025, 1, "zero", "regular4"),
                                                   (32, 2050, 4, "spectral", "regular4"), (5, 37, 2, "spectral", "path"),
                                                   (6, 50, 1, "zero", "directed"), (40, 130, 1, "zero", "ring"),
-                                                  (64, 67, 2, "spectral", "ring")])
+                                                  (64, 67, 2, "spectral", "ring"), (128, 200, 1, "zero", "ring"),
+                                                  (96, 64, 30, "spectral", "ring")])
 def test_dpsgd_one_step_and_trajectory(n, d, K, eta_mode, kind):
     rng = np.random.default_rng(n * 17 + d)
     m = _graph(kind, n)
@@ -146,7 +150,7 @@ def test_dpsgd_one_step_and_trajectory(n, d, K, eta_mode, kind):
     p = oracle_problem(m, K, eta, 0.05, a, c, 0.1, 13, 77)
     ref = []
     orc.run_dpsgd(p, x0, 8, observe=lambda st: ref.append((st.x.copy(), st.g.copy())))
-    for v in _variants(n):
+    for v in _variants(n, dpsgd_ring=kind == "ring"):
         with Session(m, d, K, eta, 0.05, a, c, x0, 0.1, 13, coord_offset=77, variant=v,
                      algorithm=B.DETAG_ALGORITHM_DPSGD) as s:
             assert B.detag_get_algorithm(s.state) == B.DETAG_ALGORITHM_DPSGD

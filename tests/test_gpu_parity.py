@@ -282,6 +282,29 @@ def test_transform_variant_is_refused_without_the_structure():
         B.detag_destroy(st)
 
 
+@pytest.mark.parametrize("n,d,K,kind", [(128, 130, 20, "ring"), (256, 67, 40, "ring"), (96, 200, 30, "directed"),
+                                         (64, 131, 3, "dense_row"), (256, 64, 196, "ring")])
+def test_circulant_kernel_with_a_dense_polynomial(n, d, K, kind):
+    """Phase lengths beyond K * bandwidth = 16 (Theorem 3's regime: K = 196 on the 256-ring) make P_K(M) a dense
+    circulant; the circulant kernel then contracts the whole ring per output block.  Also a circulant M that is
+    dense itself.  Ragged d: the last d % 64 columns run through the generic kernel in the same call."""
+    rng = np.random.default_rng(n + d + K)
+    if kind == "ring":
+        m = inputs.metropolis_weights(inputs.ring_graph(n))
+    elif kind == "directed":
+        m = inputs.directed_cycle_blend(n, 0.45, 0.35)
+    else:
+        row = rng.uniform(0.0, 1.0, n)
+        row /= row.sum()
+        m = inputs.csr_from_dense(np.stack([np.roll(row, i) for i in range(n)]))  # a full circulant, not symmetric
+    assert B.DETAG_VARIANT_RING in _variants_for(m, K)
+    eta = 0.3 if kind != "ring" else orc.spectrum(m.to_dense()).eta
+    a, c = _random_objective(rng, n, d, scale=0.1)
+    x0 = rng.standard_normal((n, d)).astype(np.float32)
+    _check_one_step(m, K, eta, 0.02, a, c, x0, 0.1, 5, j0=(1 << 32) + 3, variants=[B.DETAG_VARIANT_RING])
+    _check_trajectory(m, K, eta, 0.02, a, c, x0, 0.1, 5, steps=4, variants=[B.DETAG_VARIANT_RING])
+
+
 def test_misuse_is_reported_not_faulted():
     import torch
 
