@@ -176,17 +176,20 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
   __syncthreads();
 
   // this CTA takes slabs blockIdx.x, blockIdx.x + gridDim.x, ...
-  const long long my_slabs = blockIdx.x < p.num_slabs ? (p.num_slabs - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-  const long long num_tiles = my_slabs * NB;
+  // 32-bit bookkeeping throughout: the launcher admits d < 2^31, so slab, tile and chunk counts of a CTA fit easily,
+  // and nothing in the per-tile paths divides by a run-time value
+  const int my_slabs =
+      blockIdx.x < p.num_slabs ? static_cast<int>((p.num_slabs - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0;
+  const int num_tiles = my_slabs * NB;
   const unsigned limit = p.spin_limit;
 
   if (warp == kLoadXYWarp) {
     // ---------------------------------------------------------------- x, y chunks, each loaded once
     if (lane == 0) {
-      long long confirmed = 0;  // tiles 0 .. confirmed - 1 are known to be done with their x, y
+      int confirmed = 0;  // tiles 0 .. confirmed - 1 are known to be done with their x, y
       bool ok = true;
       // waits until every consumer warp has released all tiles up to and including `tile`
-      auto wait_released = [&](long long tile) {
+      auto wait_released = [&](int tile) {
         if (tile < confirmed) return true;
         for (int g = 0; g < kRGroups; ++g) {
           if (tile < g) continue;
@@ -197,11 +200,11 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
         confirmed = tile + 1;
         return true;
       };
-      long long Q = 0;
+      int Q = 0;
       // self test: the loads stop once the chunks of about `stall_after` tiles have gone out
       const long long stall_at = p.stall_after >= 0 ? 2 * p.stall_after : -1;
-      for (long long sl = 0; sl < my_slabs && ok; ++sl) {
-        const int half = static_cast<int>((blockIdx.x + sl * gridDim.x) * 2);
+      for (int sl = 0; sl < my_slabs && ok; ++sl) {
+        const int half = static_cast<int>((blockIdx.x + static_cast<long long>(sl) * gridDim.x) * 2);
         if (!kDense) {
           // second copy of chunk 0 for the slab's last tile; the buffer was last read by the last tile two slabs back
           if (sl >= 2) ok = wait_released((sl - 1) * NB - 1);
@@ -218,8 +221,8 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
           if (Q >= kSlots) {
             // the chunk that held this slot: position q_old of slab sl_old; its last reader is tile q_old / 2 of
             // that slab (dense mode: the slab's last tile)
-            const long long Qo = Q - kSlots, slo = Qo / CPS;
-            const int qo = static_cast<int>(Qo - slo * CPS);
+            const int Qo = Q - kSlots, slo = Qo / CPS;
+            const int qo = Qo - slo * CPS;
             const int last_reader = kDense ? NB - 1 : (qo / 2 < NB ? qo / 2 : NB - 1);
             ok = wait_released(slo * NB + last_reader);
             if (!ok) break;
@@ -233,8 +236,8 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
       }
       if (!ok) atomicExch(p.status, 1);
       // copies still in flight land in this CTA's shared memory: wait for them (bounded) before leaving
-      for (long long back = 1; back <= kSlots && back <= Q; ++back) {
-        const long long q = Q - back;
+      for (int back = 1; back <= kSlots && back <= Q; ++back) {
+        const int q = Q - back;
         bar_wait(&slot_full[q % kSlots], (q / kSlots) & 1, limit);
       }
     }
@@ -243,8 +246,8 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
   if (warp == kRSignalWarp) {
     // ---------------------------------------------------------------- publishes what has landed, strictly in order
     if (lane == 0) {
-      long long Q = 0;
-      for (long long sl = 0; sl < my_slabs; ++sl) {
+      int Q = 0;
+      for (int sl = 0; sl < my_slabs; ++sl) {
         if (!kDense) {
           if (!bar_wait(&side_full[sl & 1], (sl >> 1) & 1, limit)) {
             atomicExch(p.status, 1);
@@ -266,26 +269,28 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
   if (warp == kLoadEWarp) {
     // ---------------------------------------------------------------- g, a, c of each tile
     if (lane == 0) {
-      long long T = 0;
+      int T = 0, sl = 0, b = 0;
       bool ok = true;
       for (; T < num_tiles; ++T) {
         if (p.stall_after >= 0 && T >= p.stall_after) return;
-        const int se = static_cast<int>(T % kEStages);
+        const int se = T % kEStages;
         if (T >= kEStages) ok = bar_wait(&e_empty[se], ((T / kEStages) - 1) & 1, limit);
         if (!ok) break;
-        const long long sl = T / NB;
-        const int b = static_cast<int>(T - sl * NB);
-        const int half = static_cast<int>((blockIdx.x + sl * gridDim.x) * 2);
+        const int half = static_cast<int>((blockIdx.x + static_cast<long long>(sl) * gridDim.x) * 2);
         float* te = e_mem + static_cast<size_t>(se) * kEStageFloats;
         bar_expect_tx(&e_full[se], kEStageFloats * 4);
         rows_load(te, &maps.g, half, b * kRT, &e_full[se]);
         rows_load(te + kEArrayFloats, &maps.a, half, b * kRT, &e_full[se]);
         rows_load(te + 2 * kEArrayFloats, &maps.c, half, b * kRT, &e_full[se]);
+        if (++b == NB) {
+          b = 0;
+          ++sl;
+        }
       }
       if (!ok) {
         atomicExch(p.status, 1);
-        for (long long back = 1; back <= kEStages && back <= T; ++back) {
-          const long long q = T - back;
+        for (int back = 1; back <= kEStages && back <= T; ++back) {
+          const int q = T - back;
           bar_wait(&e_full[q % kEStages], (q / kEStages) & 1, limit);
         }
       }
@@ -294,21 +299,19 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
   }
   if (warp == kRStoreWarp) {
     if (lane == 0) {
-      for (long long T = 0; T < num_tiles; ++T) {
-        const int se = static_cast<int>(T % kEStages);
+      for (int T = 0, sl = 0, b = 0; T < num_tiles; ++T, b = (b + 1 == NB ? 0 : b + 1), sl += (b == 0 ? 1 : 0)) {
+        const int se = T % kEStages;
         if (!bar_wait(&out_ready[se], (T / kEStages) & 1, limit)) {
           atomicExch(p.status, 1);
           break;
         }
-        const long long sl = T / NB;
-        const int b = static_cast<int>(T - sl * NB);
         // rows 0..15 are read once more, into the side buffer: nothing of the slab goes out before that copy is in
         if (!kDense && b == 0 && !count_wait(side_landed, static_cast<unsigned>(sl + 1), limit)) {
           atomicExch(p.status, 1);
           break;
         }
         const float* te = e_mem + static_cast<size_t>(se) * kEStageFloats;  // now [g' | x' | y']
-        const int half = static_cast<int>((blockIdx.x + sl * gridDim.x) * 2);
+        const int half = static_cast<int>((blockIdx.x + static_cast<long long>(sl) * gridDim.x) * 2);
         rows_store(&maps.g, half, b * kRT, te);
         rows_store(&maps.xs, half, b * kRT, te + kEArrayFloats);
         if (p.mode != kModeDpsgd) rows_store(&maps.ys, half, b * kRT, te + 2 * kEArrayFloats);
@@ -347,11 +350,15 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
   }
 
   unsigned done = 0;  // tiles this group has finished
-  for (long long T = group; T < num_tiles; T += kRGroups, ++done) {
-    const long long sl = T / NB;
-    const int b = static_cast<int>(T - sl * NB);
-    const long long Qbase = sl * CPS;
-    const int se = static_cast<int>(T % kEStages);
+  // tile T = row block b of this CTA's slab number sl; Qbase = loading position of the slab's first chunk
+  int sl = group / NB, b = group % NB;
+  for (int T = group; T < num_tiles; T += kRGroups, ++done, b += kRGroups) {
+    if (b >= NB) {  // NB >= 2: at most one slab further
+      b -= NB;
+      ++sl;
+    }
+    const int Qbase = sl * CPS;
+    const int se = T % kEStages;
     // ---- the window: band mode chunks at loading positions 2b .. 2b+3 (the last one of the slab's last tile is
     // the side copy of chunk 0); dense mode all NC chunks of the slab
     const int q_first = kDense ? 0 : 2 * b;
@@ -361,41 +368,42 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
     if (lane == 0) {
       ok = count_wait(landed, static_cast<unsigned>(Qbase + q_last + 1), limit);
       if (ok && wraps) ok = count_wait(side_landed, static_cast<unsigned>(sl + 1), limit);
-      // the phases are known to be complete; these waits return at once and order this thread after the copies
-      for (int q = q_first; ok && q <= q_last; ++q)
-        ok = bar_wait(&slot_full[(Qbase + q) % kSlots], ((Qbase + q) / kSlots) & 1, limit);
-      if (ok && wraps) ok = bar_wait(&side_full[sl & 1], (sl >> 1) & 1, limit);
     }
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    // The phases are known to be complete; the waits below return at once and order the warp after the copies.
+    // One lane per barrier, all at the same time (a wait costs a few hundred cycles even when it does not wait).
+    if (ok) {
+      const int q = q_first + lane;
+      if (q <= q_last) ok = bar_wait(&slot_full[(Qbase + q) % kSlots], ((Qbase + q) / kSlots) & 1, limit);
+      if (wraps && lane == 31) ok = bar_wait(&side_full[sl & 1], (sl >> 1) & 1, limit);
+    }
+    ok = __all_sync(0xffffffffu, ok);
     if (!ok) {
       if (lane == 0) atomicExch(p.status, 1);
       return;
     }
-    const long long j = (blockIdx.x + sl * gridDim.x) * kRS + ctile * 8 + crow;  // this lane's coordinate
+    const long long j = (blockIdx.x + static_cast<long long>(sl) * gridDim.x) * kRS + ctile * 8 + crow;  // this lane's coordinate
     double cx[4][2], cy[4][2];
 #pragma unroll
     for (int t = 0; t < 4; ++t) cx[t][0] = cx[t][1] = cy[t][0] = cy[t][1] = 0.0;
-    float x_old[8];  // this lane's own rows of the old model (gradient point of Algorithm 2 as printed)
     if (!kDense) {
+      // cx accumulates P x, cy accumulates P y; the model update x' = x~ - alpha y~ happens in the tail
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {  // window chunk w: rows 32 b - 16 + 16 w ..
+      for (int w = 0; w < 4; ++w) {  // window chunk w: rows 32 b - 16 + 16 w ..; the slab's last tile ends in the side copy
         const int q = 2 * b + w;
         const float* ch = (q < CPS) ? ring_mem + static_cast<size_t>((Qbase + q) % kSlots) * kSlotFloats
                                     : side_mem + static_cast<size_t>(sl & 1) * kSlotFloats;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {  // k-step s = 4 w + i: window rows 4 s + kq
           const int s = 4 * w + i;
-          const float xv = ch[off + i * 256], yv = ch[kChunkFloats + off + i * 256];
-          if (s >= 4 && s < 12) x_old[s - 4] = xv;
-          const double by = static_cast<double>(yv);
-          // x' = P (x - alpha y) by linearity of AG_K
-          const double bx = dpsgd ? static_cast<double>(xv) : fma(-alpha, by, static_cast<double>(xv));
+          const double zx = static_cast<double>(ch[off + i * 256]);
+          const double zy = static_cast<double>(ch[kChunkFloats + off + i * 256]);
 #pragma unroll
           for (int t = 0; t < 4; ++t) {
             const int u = s - 2 * t;  // compile-time after unrolling: only the band's blocks are issued
             if (u >= 0 && u < kBandSteps) {
-              if (!dpsgd) dmma(cy[t], by, bfrag[u]);
-              dmma(cx[t], bx, bfrag[u]);
+              if (!dpsgd) dmma(cy[t], zy, bfrag[u]);
+              dmma(cx[t], zx, bfrag[u]);
             }
           }
         }
@@ -407,14 +415,7 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
         for (int i = 0; i < 4; ++i) {
           const int in_row = c * kChunkRows + 4 * i + kq;
           const float xv = ch[off + i * 256], yv = ch[kChunkFloats + off + i * 256];
-          const int m_own = in_row - b * kRT - kq;  // this lane's own output rows are b*32 + kq + 4 m
-          if (p.grad_at_start && m_own >= 0 && m_own < 32) {
-#pragma unroll
-            for (int m = 0; m < 8; ++m)
-              if (m_own == 4 * m) x_old[m] = xv;
-          }
-          const double by = static_cast<double>(yv);
-          const double bx = dpsgd ? static_cast<double>(xv) : fma(-alpha, by, static_cast<double>(xv));
+          const double by = static_cast<double>(yv), bx = static_cast<double>(xv);
 #pragma unroll
           for (int t = 0; t < 4; ++t) {
             int delta = in_row - (b * kRT + 8 * t + out_pos);  // P[out][in] = p((in - out) mod n)
@@ -425,6 +426,14 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
           }
         }
       }
+    }
+    // gradient point of Algorithm 2 as printed: this lane's own rows of the old model, still in their chunks
+    float x_old[8];
+    if (p.grad_at_start) {
+      const int q_own = kDense ? 2 * b : 2 * b + 1;
+#pragma unroll
+      for (int m = 0; m < 8; ++m)
+        x_old[m] = ring_mem[static_cast<size_t>((Qbase + q_own + (m >> 2)) % kSlots) * kSlotFloats + off + (m & 3) * 256];
     }
     __syncwarp();
     if (lane == 0) count_publish(&released[warp], done + 1);  // this warp is done with the tile's x, y chunks
@@ -439,6 +448,15 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
     float* sg = e_mem + static_cast<size_t>(se) * kEStageFloats;
     float* sa = sg + kEArrayFloats;
     float* sc = sa + kEArrayFloats;
+    // All inputs of the tail are read before anything is written back: the stores below go to the same arrays, and
+    // loads that had to stay behind them would run one element at a time.
+    float gv[8], av[8], cv[8];
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+      gv[m] = sg[off + m * 256];
+      av[m] = sa[off + m * 256];
+      cv[m] = sc[off + m * 256];
+    }
     // ---- noise: this lane's workers 32 b + kq + 4 m are position kq of the Philox quads 8 b + m, shared by the four
     // lanes of a coordinate: each draws two of the eight quads and a 4 x 4 transpose hands everybody its position
     float xi[8];
@@ -457,20 +475,24 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
       for (int m = 0; m < 8; ++m) xi[m] = 0.f;
     }
     // ---- element-wise tail on the lane's own eight elements (tile rows kq + 4 m); results replace the inputs
+    float xo[8], yo[8], go[8];
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+      const int t = m >> 1, e = m & 1;
+      // model update: x' = x~ - alpha y~ (D-PSGD: x~ - alpha g)
+      xo[m] = static_cast<float>(fma(-alpha, dpsgd ? static_cast<double>(gv[m]) : cy[t][e], cx[t][e]));
+      const float x_at = p.grad_at_start ? x_old[m] : xo[m];  // gradient point: new model, or the one the step started from
+      go[m] = fmaf(av[m], x_at - cv[m], sigma * xi[m]);
+      yo[m] = static_cast<float>((cy[t][e] - static_cast<double>(gv[m])) + static_cast<double>(go[m]));  // fold
+    }
 #pragma unroll
     for (int m = 0; m < 8; ++m) {
       const int o = off + m * 256;
-      const int t = m >> 1, e = m & 1;
-      const float gv = sg[o], av = sa[o], cv = sc[o];
-      const float xo = static_cast<float>(dpsgd ? cx[t][e] - alpha * static_cast<double>(gv) : cx[t][e]);
-      const float x_at = p.grad_at_start ? x_old[m] : xo;  // gradient point: new model, or the one the step started from
-      const float go = fmaf(av, x_at - cv, sigma * xi[m]);
-      const float yo = static_cast<float>((cy[t][e] - static_cast<double>(gv)) + static_cast<double>(go));  // fold
-      sg[o] = go;
-      sa[o] = xo;
-      sc[o] = yo;
+      sg[o] = go[m];
+      sa[o] = xo[m];
+      sc[o] = yo[m];
       if (p.y_obs != nullptr && !dpsgd)  // optional observer: the gossiped tracker, stored directly
-        p.y_obs[static_cast<long long>(b * kRT + kq + 4 * m) * p.ld + j] = static_cast<float>(cy[t][e]);
+        p.y_obs[static_cast<long long>(b * kRT + kq + 4 * m) * p.ld + j] = static_cast<float>(cy[m >> 1][m & 1]);
     }
     fence_async_shared();  // results visible to the TMA stores
     __syncwarp();
