@@ -36,6 +36,20 @@ __device__ __forceinline__ bool bar_wait(uint64_t* bar, unsigned parity, unsigne
   return false;
 }
 
+// Non-blocking test of a phase: for phases already known to be complete (through a progress counter), where the
+// caller only needs the ordering that observing the barrier gives; no suspension, no polling.
+__device__ __forceinline__ bool bar_test(uint64_t* bar, unsigned parity) {
+  unsigned done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(s_addr(bar)), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+
 // Monotonic progress counter in this CTA's shared memory (release/acquire at CTA scope), bounded wait.
 __device__ __forceinline__ void count_publish(unsigned* counter, unsigned value) {
   asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(s_addr(counter)), "r"(value) : "memory");
@@ -47,6 +61,39 @@ __device__ __forceinline__ bool count_wait(const unsigned* counter, unsigned at_
     unsigned v;
     asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
     if (v >= at_least) return true;
+    __nanosleep(100);
+  }
+  return false;
+}
+
+// The same wait with relaxed loads: for callers that follow it up with a test of the barrier the counter stands
+// for (the test is what orders them after the data); an acquiring load costs several hundred cycles each time.
+__device__ __forceinline__ bool count_wait_relaxed(const unsigned* counter, unsigned at_least, unsigned limit) {
+  const uint32_t addr = s_addr(counter);
+  for (unsigned spin = 0; spin < limit; ++spin) {
+    unsigned v;
+    asm volatile("ld.relaxed.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    if (v >= at_least) return true;
+    __nanosleep(100);
+  }
+  return false;
+}
+
+// Waits until each of `count` consecutive counters has reached `at_least`: relaxed loads issued together, one
+// acquire fence at the end (an acquiring load per counter would cost several hundred cycles each).
+__device__ __forceinline__ bool counters_wait(const unsigned* counters, int count, unsigned at_least, unsigned limit) {
+  const uint32_t addr = s_addr(counters);
+  for (unsigned spin = 0; spin < limit; ++spin) {
+    unsigned lowest = 0xffffffffu;
+    for (int k = 0; k < count; ++k) {
+      unsigned v;
+      asm volatile("ld.relaxed.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr + 4u * k) : "memory");
+      lowest = v < lowest ? v : lowest;
+    }
+    if (lowest >= at_least) {
+      asm volatile("fence.acq_rel.cta;" ::: "memory");
+      return true;
+    }
     __nanosleep(100);
   }
   return false;

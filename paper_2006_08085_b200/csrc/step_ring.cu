@@ -194,8 +194,7 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
         for (int g = 0; g < kRGroups; ++g) {
           if (tile < g) continue;
           const unsigned need = static_cast<unsigned>((tile - g) / kRGroups + 1);  // tiles of group g among 0 .. tile
-          for (int w = 0; w < kRGroupWarps; ++w)
-            if (!count_wait(&released[g * kRGroupWarps + w], need, limit)) return false;
+          if (!counters_wait(&released[g * kRGroupWarps], kRGroupWarps, need, limit)) return false;
         }
         confirmed = tile + 1;
         return true;
@@ -359,6 +358,25 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
     }
     const int Qbase = sl * CPS;
     const int se = T % kEStages;
+    const long long j = (blockIdx.x + static_cast<long long>(sl) * gridDim.x) * kRS + ctile * 8 + crow;  // this lane's coordinate
+    // The normals of this tile need no data: they are drawn first, while the tile's chunks may still be on their way.
+    // This lane's workers 32 b + kq + 4 m are position kq of the Philox quads 8 b + m, shared by the four
+    // lanes of a coordinate: each draws two of the eight quads and a 4 x 4 transpose hands everybody its position
+    float xi[8];
+    if (noisy) {
+      const unsigned long long jn = static_cast<unsigned long long>(p.coord_offset + j);
+#pragma unroll
+      for (int hq = 0; hq < 2; ++hq) {
+        float v[4];
+        normal_quad(p.seed_lo, p.seed_hi, jn, static_cast<uint32_t>(8 * b + 4 * hq + kq), p.t_noise, v);
+        transpose_over_kq(v, kq);  // v[i]: position kq of quad 8 b + 4 hq + i
+#pragma unroll
+        for (int i = 0; i < 4; ++i) xi[4 * hq + i] = v[i];
+      }
+    } else {
+#pragma unroll
+      for (int m = 0; m < 8; ++m) xi[m] = 0.f;
+    }
     // ---- the window: band mode chunks at loading positions 2b .. 2b+3 (the last one of the slab's last tile is
     // the side copy of chunk 0); dense mode all NC chunks of the slab
     const int q_first = kDense ? 0 : 2 * b;
@@ -366,23 +384,27 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
     const bool wraps = !kDense && 2 * b + 3 >= CPS;
     bool ok = true;
     if (lane == 0) {
-      ok = count_wait(landed, static_cast<unsigned>(Qbase + q_last + 1), limit);
-      if (ok && wraps) ok = count_wait(side_landed, static_cast<unsigned>(sl + 1), limit);
+      ok = count_wait_relaxed(landed, static_cast<unsigned>(Qbase + q_last + 1), limit);
+      if (ok && wraps) ok = count_wait_relaxed(side_landed, static_cast<unsigned>(sl + 1), limit);
     }
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-    // The phases are known to be complete; the waits below return at once and order the warp after the copies.
-    // One lane per barrier, all at the same time (a wait costs a few hundred cycles even when it does not wait).
+    // The phases are known to be complete: a non-blocking test per barrier (one lane each, all at once) orders the
+    // warp after the copies; should a test ever fail, the bounded wait takes over.
     if (ok) {
       const int q = q_first + lane;
-      if (q <= q_last) ok = bar_wait(&slot_full[(Qbase + q) % kSlots], ((Qbase + q) / kSlots) & 1, limit);
-      if (wraps && lane == 31) ok = bar_wait(&side_full[sl & 1], (sl >> 1) & 1, limit);
+      if (q <= q_last) {
+        uint64_t* bar = &slot_full[(Qbase + q) % kSlots];
+        const unsigned parity = ((Qbase + q) / kSlots) & 1;
+        if (!bar_test(bar, parity)) ok = bar_wait(bar, parity, limit);
+      }
+      if (wraps && lane == 31 && !bar_test(&side_full[sl & 1], (sl >> 1) & 1))
+        ok = bar_wait(&side_full[sl & 1], (sl >> 1) & 1, limit);
     }
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) {
       if (lane == 0) atomicExch(p.status, 1);
       return;
     }
-    const long long j = (blockIdx.x + static_cast<long long>(sl) * gridDim.x) * kRS + ctile * 8 + crow;  // this lane's coordinate
     double cx[4][2], cy[4][2];
 #pragma unroll
     for (int t = 0; t < 4; ++t) cx[t][0] = cx[t][1] = cy[t][0] = cy[t][1] = 0.0;
@@ -456,23 +478,6 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
       gv[m] = sg[off + m * 256];
       av[m] = sa[off + m * 256];
       cv[m] = sc[off + m * 256];
-    }
-    // ---- noise: this lane's workers 32 b + kq + 4 m are position kq of the Philox quads 8 b + m, shared by the four
-    // lanes of a coordinate: each draws two of the eight quads and a 4 x 4 transpose hands everybody its position
-    float xi[8];
-    if (noisy) {
-      const unsigned long long jn = static_cast<unsigned long long>(p.coord_offset + j);
-#pragma unroll
-      for (int hq = 0; hq < 2; ++hq) {
-        float v[4];
-        normal_quad(p.seed_lo, p.seed_hi, jn, static_cast<uint32_t>(8 * b + 4 * hq + kq), p.t_noise, v);
-        transpose_over_kq(v, kq);  // v[i]: position kq of quad 8 b + 4 hq + i
-#pragma unroll
-        for (int i = 0; i < 4; ++i) xi[4 * hq + i] = v[i];
-      }
-    } else {
-#pragma unroll
-      for (int m = 0; m < 8; ++m) xi[m] = 0.f;
     }
     // ---- element-wise tail on the lane's own eight elements (tile rows kq + 4 m); results replace the inputs
     float xo[8], yo[8], go[8];
