@@ -83,7 +83,6 @@ bool dense_variant_available(int n);  // n <= kMaxDenseWorkers and the driver of
 bool build_maps_mma(const StepParams& p, TensorMapSet* maps);
 int launch_step_mma(StepParams p, const TensorMapSet& maps, int sm_count, cudaStream_t stream);       // n <= 32
 int launch_step_mma_many(StepParams p, const TensorMapSet& maps, int sm_count, cudaStream_t stream);  // p.steps steps
-bool band_variant_available(int n, int half_band);  // circulant band kernel: n % 32 == 0, n >= 64, half-band <= 16
 bool dense_window_available(int n);                // the band kernel's dense mode: 32 < n <= 64
 bool build_maps_band(const StepParams& p, TensorMapSet* maps);
 int launch_step_band(StepParams p, const TensorMapSet& maps, const double* band /* null: dense mode */, int sm_count,

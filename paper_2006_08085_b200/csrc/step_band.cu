@@ -1,43 +1,25 @@
-// DeTAG step for circulant gossip matrices (rings) with many workers: banded polynomial on the FP64 tensor path.
+// DeTAG step with the dense polynomial for 32 < n <= 64 workers (any gossip matrix) on the FP64 tensor path.
 //
-// For a circulant M (every row is the previous one shifted by one: the ring with uniform weights, the paper's
-// Metropolis ring and its slack matrices) the K-round accelerated gossip AG_K(z) = P z has a circulant
-// P = P_K(M) whose row is a band: P[i][j] = p((j - i) mod n), p(delta) = 0 for |delta| > K * (bandwidth of M).
-// The dense product needs n multiply-adds per element, the K sparse rounds 3K dependent ones; the band needs
-// 2K+1, and it can be applied to a block of output rows from a window of input rows:
-//     out rows [R, R+32)  <-  window rows [R-16, R+48)   (mod n),   half-band <= 16.
-// Per 8-coordinate tile that is, for each of the four 8-row output blocks t, the ten 4-row window steps
-// s = 2t .. 2t+9 (all other blocks of the 32 x 64 band matrix are zero): 80 float64 MMAs (m8n8k4) for the
-// tracker and the model together, and because P is circulant the A fragment depends on s - 2t only:
-// ten doubles per lane, kept in registers, for every tile of the run.
+// AG_K(z) = P z with P = P_K(M) built by the host in float64.  One unit of work ("tile") is 32 output rows x 64
+// coordinates; its window is all 64 rows (rows >= n are zero-filled by the loads), every one of the 16 x 4 blocks of
+// the 32 x 64 slice of P is issued (128 float64 MMAs m8n8k4 per 8-coordinate tile for tracker and model together)
+// and the A fragments come from shared memory (32 KB for the two slices).
 //
-// A CTA owns whole slabs of 64 coordinates and walks the n/32 row blocks of a slab in order; one unit of work
-// ("tile") is 32 output rows x 64 coordinates.  Warp roles, mbarrier pipeline, padded TMA input tiles (box =
-// row pitch), dense output tile + TMA tile stores, tail inputs in registers and the stage handed back before
-// the tail: as in the dense kernel for n <= 32.  The window rows wrap around the ring, so the x, y windows are
-// fetched as four 16-row boxes each at row (R - 16 + 16 q) mod n; g, a, c are needed for the 32 output rows only.
-// The halo rows are read twice (once per neighbouring block); the second read comes from L2.
+// A CTA owns whole slabs of 64 coordinates and walks the two row blocks of a slab in order.  Warp roles, mbarrier
+// pipeline, padded TMA input tiles (box = row pitch), dense output tile + TMA tile stores, tail inputs in registers
+// and the stage handed back before the tail: as in the dense kernel for n <= 32.  The x, y window is fetched as four
+// 16-row boxes; g, a, c are needed for the 32 output rows only.  The window is read twice (once per row block);
+// the second read comes from L2.
 //
-// The step updates x and y in place, and a tile's window contains rows that the neighbouring row blocks
-// overwrite.  Two rules keep every window on the old values:
-//   * the results of row block b are stored only after the window of block b+1 (which contains the last 16
-//     rows of block b) has landed in shared memory: a signalling thread publishes a "tiles landed" counter,
-//     and the storing thread (and the warps that write the d % 4 tail columns directly) wait for it;
-//   * the window of the last block ends with rows 0..15, which block 0 has overwritten long before: those
-//     rows are fetched into a side buffer together with block 0's window (before anything of the slab is
-//     stored) and the last block reads them from there.
-// Blocks further apart share no rows (n >= 64), and different slabs share no coordinates.
+// The step updates x and y in place, and the second tile's window contains the rows the first tile overwrites: the
+// results of row block 0 are stored only after the window of block 1 has landed in shared memory (a signalling
+// thread publishes a "tiles landed" counter; the storing thread, and the warps that write the d % 4 tail columns
+// directly, wait for it).  Different slabs share no coordinates.
 //
-// Dense mode (template flag): for 32 < n <= 64 the same machinery applies the full polynomial P_K(M) of any gossip
-// matrix.  The window is then simply rows 0..63 (all workers; rows >= n are zero-filled by the loads) for both
-// row blocks, every one of the 16 x 4 blocks of the 32 x 64 slice of P is issued (128 MMAs per tile), and the A
-// fragments come from shared memory (32 KB for the two slices) instead of ten registers.  No rows wrap, so the
-// side buffer is idle; the first in-place rule is all that is needed.
-//
-// Output rows are the natural blocks 8t + r (a permuted block would widen the band), so the four workers of
-// one Philox call sit in four lanes: each lane draws the calls of one block and a 4 x 4 transpose over those
-// lanes (two shuffle stages) hands every lane its own workers' normals.
-// Every mbarrier wait is bounded; a wait that gives up sets the status word and the CTA winds down.
+// Output rows are the natural blocks 8t + r, so the four workers of one Philox call sit in four lanes: each lane
+// draws the calls of one block and a 4 x 4 transpose over those lanes (two shuffle stages) hands every lane its
+// own workers' normals.  Every mbarrier wait is bounded; a wait that gives up sets the status word and the CTA
+// winds down.  (Circulant matrices with n >= 64 have their own kernel, step_ring.cu; tori step_torus.cu.)
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -67,7 +49,6 @@ constexpr int kProducerWarp = kConsumerWarps, kStoreWarp = kConsumerWarps + 1, k
 constexpr int kThreads = (kConsumerWarps + 3) * 32;
 constexpr int kSideFloats = 2 * kHalo * kPitchXY;  // rows 0..15 of x and y, kept for the slab's last row block
 constexpr int kOutFloats = 3 * kR * kS;
-constexpr int kBandSteps = 10;     // 4-row window steps that meet an 8-row output block: (2*16 + 8) / 4
 constexpr size_t kSmemBytes =
     static_cast<size_t>(kStages) * kStageBytes + 2 * kSideFloats * 4 + kWarpGroups * kOutFloats * 4 + 128;  // + barriers, counters
 constexpr int kDenseFragBytes = 2 * (kW / 4) * 4 * 32 * 8;  // dense mode: [row block][window step][t][lane] doubles
@@ -80,10 +61,6 @@ struct BandMaps {
 };
 
 static_assert(sizeof(BandMaps) <= sizeof(TensorMapSet), "tensor map storage");
-
-struct BandCoef {
-  double p[2 * kHalo + 1];  // p[delta + kHalo] = P[i][(i + delta) mod n]
-};
 
 // 4 x 4 transpose over the four lanes {lane ^ 0, 4, 8, 12} (lane bits 2 and 3): lane with index q = (lane >> 2) & 3
 // gives row q = v[0..3] and receives column q.
@@ -99,9 +76,9 @@ __device__ __forceinline__ void transpose4(float (&v)[4], int q) {
   if (b1) { v[0] = r0; v[1] = r1; } else { v[2] = r0; v[3] = r1; }
 }
 
-template <bool kDense>
 __global__ void __launch_bounds__(kThreads, 1)
-step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, const __grid_constant__ BandCoef coef) {
+step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps) {
+  constexpr bool kDense = true;  // the whole 64-row window, every block of P
   // No static shared memory: the dynamic array starts at the CTA's shared window; its alignment is checked.
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* stage_mem = reinterpret_cast<float*>(smem_raw);
@@ -257,15 +234,6 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
   float* ob = out_mem + group * kOutFloats;
   const int cl = mtile * 8;
   const long long d_tma = p.d & ~3LL;
-  // A fragment of window step u = s - 2t: element [r][kq] = p(4u + kq - r - 16); the same for every block and tile
-  double afrag[kDense ? 1 : kBandSteps];
-  if (!kDense) {
-#pragma unroll
-    for (int u = 0; u < kBandSteps; ++u) {
-      const int delta = 4 * u + kq - r - kHalo;
-      afrag[u] = (delta >= -kHalo && delta <= kHalo) ? coef.p[delta + kHalo] : 0.0;
-    }
-  }
   const int pos = r & 3, half = r >> 2;  // this lane's worker is number `pos` of its Philox quad
 
   // 32-bit bookkeeping: the launcher admits this kernel only for d < 2^31, so tile and slab counts fit easily
@@ -324,17 +292,9 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
         const double bx = fma(-alpha, by, static_cast<double>(sx[src + (side ? side_dx : 0)]));
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-          if (kDense) {
-            const double a = frag[((rb * (kW / 4) + ws) * 4 + t) * 32 + lane];
-            dmma(cy[t], a, by);
-            dmma(cx[t], a, bx);
-          } else {
-            const int u = ws - 2 * t;  // compile-time after unrolling: only the band's blocks are issued
-            if (u >= 0 && u < kBandSteps) {
-              dmma(cy[t], afrag[u], by);
-              dmma(cx[t], afrag[u], bx);
-            }
-          }
+          const double a = frag[((rb * (kW / 4) + ws) * 4 + t) * 32 + lane];
+          dmma(cy[t], a, by);
+          dmma(cx[t], a, bx);
         }
       }
       // the tail's inputs move to registers so that the stage can be refilled while the tail runs
@@ -427,10 +387,6 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps, cons
 
 }  // namespace
 
-bool band_variant_available(int n, int half_band) {
-  return n % kR == 0 && n >= kW && n <= kMaxWorkers && half_band <= kHalo && encode_tiled_fn() != nullptr;
-}
-
 bool dense_window_available(int n) { return n > kR && n <= kW && encode_tiled_fn() != nullptr; }
 
 bool dense_variant_available(int n) { return n >= 1 && n <= kMaxDenseWorkers && encode_tiled_fn() != nullptr; }
@@ -449,22 +405,18 @@ bool build_maps_band(const StepParams& p, TensorMapSet* out) {
   return true;
 }
 
-// band == nullptr: dense mode (32 < n <= 64, p.poly holds P_K(M)); otherwise the circulant band of 2*16+1 entries,
-// p(delta) at index delta + 16.
+// 32 < n <= 64, p.poly holds P_K(M); `band` must be null (kept for the launcher's signature).
 int launch_step_band(StepParams p, const TensorMapSet& maps, const double* band, int sm_count, cudaStream_t stream) {
-  if (p.mode != kModeDetag) return static_cast<int>(cudaErrorInvalidValue);
-  BandCoef coef;
-  const bool dense = band == nullptr;
-  for (int k = 0; k < 2 * kHalo + 1; ++k) coef.p[k] = dense ? 0.0 : band[k];
+  if (p.mode != kModeDetag || band != nullptr) return static_cast<int>(cudaErrorInvalidValue);
   p.S = kS;
   p.num_slabs = (p.d + kS - 1) / kS;
-  auto kernel = dense ? step_band_kernel<true> : step_band_kernel<false>;
-  const size_t smem = kSmemBytes + (dense ? kDenseFragBytes : 0);
+  auto kernel = step_band_kernel;
+  const size_t smem = kSmemBytes + kDenseFragBytes;
   const int e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), static_cast<int>(smem));
   if (e != 0) return e;
   const long long grid = p.num_slabs < sm_count ? p.num_slabs : sm_count;
   if (grid <= 0) return 0;
-  kernel<<<static_cast<unsigned>(grid), kThreads, smem, stream>>>(p, *reinterpret_cast<const BandMaps*>(maps.bytes), coef);
+  kernel<<<static_cast<unsigned>(grid), kThreads, smem, stream>>>(p, *reinterpret_cast<const BandMaps*>(maps.bytes));
   return static_cast<int>(cudaGetLastError());
 }
 
