@@ -184,6 +184,24 @@ int detag_get_algorithm(const detag_state* s, int* algorithm);
 int detag_set_gradient_source(detag_state* s, int source, const float* g_new);
 
 /*
+ * Stochastic gradient of the zero-chain objective of the paper's lower-bound construction (proof of Theorem 1:
+ * the equation defining the base function fhat, and "Setting 1": every worker holds fhat, rescaled as
+ * f(x) = (L lambda^2 / l_1) fhat(x / lambda); the oracle multiplies the partial derivatives beyond the progress of
+ * x - its last non-zero coordinate - by z / p with z ~ Bernoulli(p), one draw per worker and step):
+ *     g_out[i][j] = gain * d_j fhat(x_i / lambda) * (j > prog(x_i) ? z_i / p : 1)          gain = L lambda / l_1
+ *     fhat(u) = sum_{i=0}^{d-1} [Psi(-u_i) Phi(-u_{i+1}) - Psi(u_i) Phi(u_{i+1})],  u_0 := 1,
+ *     Psi(z) = exp(1 - 1/(2z-1)^2) for z > 1/2 (else 0),  Phi(z) = sqrt(e) int_{-inf}^z exp(-t^2/2) dt.
+ * The chain runs over all d coordinates of a worker, which are coupled to their neighbours: unlike the diagonal
+ * objective this gradient cannot be evaluated shard by shard.  z_i is a pure function of (seed, t, i).
+ * x, g_out: device, [n][ld] float32 (may not alias); scratch: device, n int32 (per-worker progress, overwritten).
+ * Meant to be used with detag_set_gradient_source(DETAG_GRADIENT_EXTERNAL): write g_out = the registered array
+ * before each detag_step.  Asynchronous on `stream`.  No detag_state is involved.
+ * Errors: ARG (null pointers, ld < d, lambda <= 0, p outside (0, 1], t < 0), UNSUPPORTED (n > 1024, d >= 2^31), CUDA.
+ */
+int detag_zero_chain_gradient(int n, int64_t d, int64_t ld, const float* x, float* g_out, double lambda, double gain,
+                              double p, uint64_t seed, int64_t t, int32_t* scratch, void* stream);
+
+/*
  * Phase length of Theorem 3: R = max(1/2 ln n, 1/2 ln(varsigma0_sq * T / delta_L)) / sqrt(1 - lambda),
  * rounded up to a whole number of gossip rounds, at least 1.  lambda as returned by detag_spectral,
  * varsigma0_sq the bound on the gradient dissimilarity at the origin (Section "Setting"), T the

@@ -69,6 +69,8 @@ SIGNATURES = {
     "detag_set_gradient_source": (ctypes.c_int, [_P, ctypes.c_int, _P]),
     "detag_debug_inject_stall": (ctypes.c_int, [_P, ctypes.c_int64, ctypes.c_uint32]),
     "detag_debug_expire_wait": (ctypes.c_int, [_P, ctypes.c_uint32, _P]),
+    "detag_zero_chain_gradient": (ctypes.c_int, [ctypes.c_int, ctypes.c_int64, ctypes.c_int64, _P, _P, ctypes.c_double,
+                                                 ctypes.c_double, ctypes.c_double, ctypes.c_uint64, ctypes.c_int64, _P, _P]),
     "detag_phase_length": (ctypes.c_int, [ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_double,
                                           ctypes.c_double, ctypes.POINTER(ctypes.c_int)]),
     "detag_init": (ctypes.c_int, [_P, _P]),
@@ -220,6 +222,15 @@ def detag_debug_inject_stall(state, after_tiles: int, poll_limit: int = 2048) ->
 
 def detag_debug_expire_wait(state, polls: int, stream=None) -> None:
     _check(lib().detag_debug_expire_wait(state, int(polls), _stream_handle(stream)), "detag_debug_expire_wait", state)
+
+
+def detag_zero_chain_gradient(n: int, d: int, ld: int, x, g_out, lam: float, gain: float, p: float, seed: int, t: int,
+                              scratch, stream=None) -> None:
+    """Bernoulli-progress gradient oracle of the zero-chain objective (proof of Theorem 1) into g_out; scratch is a
+    device int32 tensor with n entries."""
+    _check(lib().detag_zero_chain_gradient(int(n), int(d), int(ld), _dev_ptr(x), _dev_ptr(g_out), float(lam), float(gain),
+                                           float(p), int(seed), int(t), _dev_ptr(scratch), _stream_handle(stream)),
+           "detag_zero_chain_gradient")
 
 
 def detag_phase_length(n: int, lam: float, varsigma0_sq: float = 0.0, T: float = 0.0, delta_L: float = 1.0) -> int:
