@@ -40,6 +40,7 @@ BYTES_PER_WC = 32  # read x, y, g, a, c + write x, y, g, float32 each: the fused
 KERNEL_SOURCES = {
     "mma": ("step_mma.cu", "mma_common.cuh", "pipeline.cuh", "noise.cuh"),
     "band": ("step_band.cu", "pipeline.cuh", "noise.cuh"),
+    "ring": ("step_ring.cu", "pipeline.cuh", "noise.cuh"),
     "csr": ("step_csr.cu", "noise.cuh"),
     "torus": ("step_torus.cu", "torus_basis.h", "pipeline.cuh", "noise.cuh"),
 }
@@ -49,8 +50,8 @@ MEASURED_TRAFFIC = {
 
 # Float64 multiply-adds per worker-coordinate on the FP64 pipe (both contractions, padded shapes) and that
 # pipe's peak: 64 multiply-adds per clock and SM (measured: 61 with m8n8k4 MMAs from 16 warps) x 148 SMs x max clock.
-FP64_FMA_PER_WC = {("mma", "dense"): 64, ("band", "ring"): 80, ("band", "dense"): 128,
-                   ("torus", "torus8"): 40, ("torus", "torus4"): 28}
+FP64_FMA_PER_WC = {("mma", "dense"): 64, ("ring", "band"): 80, ("band", "dense"): 128,
+                   ("torus", "torus8"): 26, ("torus", "torus4"): 28}
 VARIANT_NAMES = {1: "csr", 2: "dense", 3: "ring", 4: "torus"}
 FP64_FMA_PER_CLK_SM = 64
 SM_COUNT = 148
@@ -60,7 +61,7 @@ def kernel_key(variant: str, n: int):
     if variant == "dense":
         return ("mma", "dense") if n <= 32 else ("band", "dense")
     if variant == "ring":
-        return ("band", "ring")
+        return ("ring", "band")
     if variant == "csr":
         return ("csr", "rounds")
     if variant == "torus":
@@ -195,6 +196,7 @@ class ClockSampler(threading.Thread):
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop_evt = threading.Event()
+        self.ready = threading.Event()  # set once the first sample is in (NVML start-up can take a while)
         self.error = None
 
     def run(self):
@@ -209,9 +211,11 @@ class ClockSampler(threading.Thread):
                 for bit, name in self.REASONS.items():
                     if mask & bit:
                         self.reasons.add(name)
+                self.ready.set()
                 time.sleep(self.period)
         except Exception as exc:  # NVML missing: report it, the timing itself is unaffected
             self.error = repr(exc)
+            self.ready.set()
 
     def stop(self):
         self._stop_evt.set()
@@ -282,6 +286,50 @@ def time_config(name: str, dev, args) -> dict:
     if key in FP64_FMA_PER_WC:
         out["fp64_fma_per_wc"] = FP64_FMA_PER_WC[key]
         out["fp64_pipe_frac"] = FP64_FMA_PER_WC[key] * out["value"] / (FP64_FMA_PER_CLK_SM * SM_COUNT * 1965e6)
+    return out
+
+
+def theorem3_regime(dev, args) -> dict:
+    """cfg4's 256-ring at the configuration's K = 16 and at Theorem 3's phase length (K = 196, where the gossip
+    polynomial is a dense circulant), on a 200,000-coordinate cut: step time and the consensus error per
+    worker-coordinate after every step (it grows at K = 16 and contracts at Theorem 3's K)."""
+    import dataclasses
+
+    import torch
+
+    from paper_2006_08085_b200 import binding as B
+    from paper_2006_08085_b200.session import Session
+
+    base = inputs.CONFIGS["cfg4"].with_d(200_000)
+    gm = inputs.gossip_matrix(base)
+    lam = B.detag_spectral(gm.n, gm.row_ptr, gm.col_idx, gm.vals)[2]
+    k_thm = B.detag_phase_length(gm.n, lam)
+    a, c, x0 = inputs.objective_data(base, threads=min(32, os.cpu_count() or 1))
+    out = {"workload": "cfg4 ring, d = 200,000", "lambda": lam, "runs": []}
+    stream = torch.cuda.current_stream(dev)
+    for K in (base.K, k_thm):
+        cfg = dataclasses.replace(base, K=K)
+        s = Session(gm, cfg.d, cfg.K, float("nan"), cfg.alpha, a, c, x0, cfg.sigma, cfg.seed, device=str(dev))
+        s.init()
+        ce = [s.consensus_error() / cfg.wc]
+        steps = 10
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ms = 0.0
+        for _ in range(steps):
+            e0.record(stream)
+            B.detag_step(s.state, stream)
+            e1.record(stream)
+            torch.cuda.synchronize(dev)
+            ms += e0.elapsed_time(e1)
+            ce.append(s.consensus_error() / cfg.wc)
+        s.status()
+        out["runs"].append({"K": K, "variant": VARIANT_NAMES.get(B.detag_get_variant(s.state), "other"),
+                            "ms_per_step": ms / steps, "value": cfg.wc / (ms / steps * 1e-3), "unit": UNIT,
+                            "fp64_fma_per_wc": 80 if K == base.K else 2 * cfg.n,
+                            "consensus_error_per_wc_by_step": ce})
+        s.close()
+        del s
+    torch.cuda.empty_cache()
     return out
 
 
@@ -364,7 +412,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
 
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
-    time.sleep(0.05)
+    sampler.ready.wait(5.0)
     events = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     events[0].record(stream)
     for k in range(args.steps):
@@ -519,6 +567,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         if world == 1 and not args.no_per_config:
             line["per_config"] = [time_config(name, dev, args) for name in sorted(inputs.CONFIGS)
                                   if name != cfg.name or args.d]
+            line["theorem3_regime"] = theorem3_regime(dev, args)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(inputs.CONFIGS[args.config], 10.0)
         print(json.dumps(line), flush=True)
