@@ -333,6 +333,43 @@ def theorem3_regime(dev, args) -> dict:
     return out
 
 
+def general_graph(dev, args) -> dict:
+    """A graph none of the structured kernels takes - 100 workers on a seeded random 4-regular graph, K = 6,
+    d = 2,000,000 - through the generic rounds kernel: its step time and roofline fraction."""
+    import torch
+
+    from paper_2006_08085_b200 import binding as B
+    from paper_2006_08085_b200.session import Session
+
+    n, d, K = 100, 2_000_000, 6
+    gm = inputs.metropolis_weights(inputs.random_regular4_graph(n, 7))
+    s = Session(gm, d, K, float("nan"), 0.001, None, None, None, 0.1, 7, device=str(dev))
+    gen = torch.Generator(device=dev).manual_seed(7)
+    s.a.uniform_(0.5, 2.0, generator=gen)  # objective data drawn on the device: this leg times the kernel only
+    s.c.normal_(generator=gen)
+    stream = torch.cuda.current_stream(dev)
+    s.init()
+    for _ in range(3):
+        B.detag_step(s.state, stream)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(10):
+        B.detag_step(s.state, stream)
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    s.status()
+    ms = e0.elapsed_time(e1) / 10
+    variant = VARIANT_NAMES.get(B.detag_get_variant(s.state), "other")
+    s.close()
+    del s
+    torch.cuda.empty_cache()
+    peak, _ = measured_peak_gbs()
+    gbs = BYTES_PER_WC * n * d / (ms * 1e-3) / 1e9
+    return {"workload": "100 workers, random 4-regular graph (Metropolis weights), d = 2,000,000, K = 6", "variant": variant,
+            "ms_per_step": ms, "value": n * d / (ms * 1e-3), "unit": UNIT, "achieved_gbs": gbs,
+            "frac_of_measured_peak": gbs / peak, "frac_of_8TBps_nominal": gbs / 8000.0}
+
+
 def run_host_only(args, rank: int, world: int) -> None:
     """The multi-rank plumbing without a GPU: the ranks meet over gloo, work out their shards and reduce the two
     scalars the real run reduces (slowest rank's time, sum of the shards' consensus errors)."""
@@ -568,6 +605,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
             line["per_config"] = [time_config(name, dev, args) for name in sorted(inputs.CONFIGS)
                                   if name != cfg.name or args.d]
             line["theorem3_regime"] = theorem3_regime(dev, args)
+            line["general_graph"] = general_graph(dev, args)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(inputs.CONFIGS[args.config], 10.0)
         print(json.dumps(line), flush=True)

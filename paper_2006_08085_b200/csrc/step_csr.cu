@@ -1,17 +1,20 @@
-// Generic DeTAG step kernel: K accelerated-gossip rounds as neighbour-indexed sums over the CSR
-// rows of M, on a coordinate slab of all n workers that is staged once in shared memory.
+// Generic DeTAG step kernel: K accelerated-gossip rounds as neighbour-indexed sums over the CSR rows of M, on a
+// coordinate slab of all n workers that is staged once in shared memory (any graph, any K, n <= 1024).
 //
-// Per slab of S coordinates a CTA
-//   1. loads x and y for all n workers, widened to float64, into the "current" and "previous"
-//      buffers (Algorithm 3 starts with z_{-1} = z_0),
-//   2. runs K rounds  z_{r+1,i} = (1+eta) sum_j M[i][j] z_{r,j} - eta z_{r-1,i}  for both arrays;
-//      the new value overwrites the previous-round slot of the same element, so two buffers
-//      per array suffice and one barrier per round orders them,
-//   3. finishes the step element-wise (Algorithm 2): x' = x~ - alpha y~, the stochastic gradient
-//      g' = a (x' - c) + sigma xi at the new model, and the tracker fold y' = y~ + g' - g with the
-//      float32 value of g' that is stored, so that the stored tracker telescopes exactly
-//      against the stored gradients.
-// All on-chip arithmetic is float64; each result is rounded once when it is stored.
+// A thread owns one worker and four consecutive coordinates of the slab for the whole step.  Per slab
+//   1. it loads its x and y (one 16-byte load each), widens them to float64, keeps them as the "previous" values of
+//      Algorithm 3 (z_{-1} = z_0) in registers and publishes them in the shared slab;
+//   2. K rounds  z_{r+1,i} = (1+eta) sum_j M[i][j] z_{r,j} - eta z_{r-1,i}  for both arrays: the neighbour values are
+//      32-byte reads from the shared slab (the row's column indices and weights are read once per round and serve
+//      all eight values), the thread's own previous values never leave its registers; a barrier separates reading
+//      a round's inputs from overwriting them, so one slab buffer per array suffices;
+//   3. it finishes the step element-wise (Algorithm 2): x' = x~ - alpha y~, the stochastic gradient
+//      g' = a (x' - c) + sigma xi at the new model (the four workers of a Philox call sit in four neighbouring lanes:
+//      each lane draws one of the four coordinates and a 4 x 4 transpose hands everybody its own row), and the
+//      tracker fold y' = y~ + g' - g with the float32 value of g' that is stored, so that the stored tracker
+//      telescopes exactly against the stored gradients; a, c, g are 16-byte loads, x', y', g' 16-byte stores.
+// All on-chip arithmetic is float64; each result is rounded once when it is stored.  What bounds the kernel is the
+// shared-memory traffic of step 2: 8 bytes per multiply-add.
 //
 // Modes: with caller-written gradients step 1 also applies Algorithm 2's tracker update, y + g_new - g_old, and
 // step 3 stores the gossiped tracker and copies g_new over g_old instead of evaluating a gradient; in D-PSGD
@@ -25,121 +28,218 @@ namespace detag {
 
 namespace {
 
-constexpr int kCsrThreads = 256;
+constexpr int kCsrThreads = 1024;
+constexpr int kCsrPad = 4;  // doubles of padding per slab row: neighbouring rows start 8 banks apart
 
-__host__ __device__ inline size_t csr_smem_bytes(int n, int nnz, int S) {
-  // four slab buffers (x/y, current/previous) + values + row pointers + columns
-  return static_cast<size_t>(4) * n * S * sizeof(double) + static_cast<size_t>(nnz) * sizeof(double) +
-         static_cast<size_t>(n + 1 + nnz) * sizeof(int32_t);
+__host__ __device__ inline size_t csr_smem_bytes(int n, int nnz, int S, bool tables) {
+  // the x and y slabs + (if they fit) values, row pointers and columns
+  return static_cast<size_t>(2) * n * (S + kCsrPad) * sizeof(double) +
+         (tables ? static_cast<size_t>(nnz) * sizeof(double) + static_cast<size_t>(n + 1 + nnz) * sizeof(int32_t) : 0);
 }
 
-__global__ void __launch_bounds__(kCsrThreads) step_csr_kernel(const StepParams p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int n = p.n, S = p.S, NS = n * S, tid = threadIdx.x;
-  double* cur_x = reinterpret_cast<double*>(smem_raw);
-  double* cur_y = cur_x + NS;
-  double* prv_x = cur_y + NS;
-  double* prv_y = prv_x + NS;
-  double* s_val = prv_y + NS;
-  int32_t* s_row = reinterpret_cast<int32_t*>(s_val + p.nnz);
-  int32_t* s_col = s_row + (n + 1);
+// 4 x 4 transpose over the four lanes that share a coordinate group (lane bits 0 and 1).
+__device__ __forceinline__ void transpose_rows(float (&v)[4], int r4) {
+  const bool b0 = (r4 & 1) != 0, b1 = (r4 & 2) != 0;
+  float s0 = b0 ? v[0] : v[1], s1 = b0 ? v[2] : v[3];
+  float r0 = __shfl_xor_sync(0xffffffffu, s0, 1), r1 = __shfl_xor_sync(0xffffffffu, s1, 1);
+  if (b0) { v[0] = r0; v[2] = r1; } else { v[1] = r0; v[3] = r1; }
+  s0 = b1 ? v[0] : v[2];
+  s1 = b1 ? v[1] : v[3];
+  r0 = __shfl_xor_sync(0xffffffffu, s0, 2);
+  r1 = __shfl_xor_sync(0xffffffffu, s1, 2);
+  if (b1) { v[0] = r0; v[1] = r1; } else { v[2] = r0; v[3] = r1; }
+}
 
-  for (int k = tid; k < p.nnz; k += kCsrThreads) {
-    s_val[k] = p.vals[k];
-    s_col[k] = p.col_idx[k];
+__device__ __forceinline__ void load4(const float* base, long long off, long long j, long long d, float (&v)[4]) {
+  if (j + 3 < d) {
+    const float4 t = *reinterpret_cast<const float4*>(base + off);
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  } else {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = j + e < d ? base[off + e] : 0.f;
   }
-  for (int k = tid; k <= n; k += kCsrThreads) s_row[k] = p.row_ptr[k];
+}
 
-  const double one_plus_eta = 1.0 + p.eta, eta = p.eta, alpha = p.alpha, sigma = p.sigma;
-  const int nq = (n + 3) >> 2;
+__device__ __forceinline__ void store4(float* base, long long off, long long j, long long d, const float (&v)[4]) {
+  if (j + 3 < d) {
+    *reinterpret_cast<float4*>(base + off) = make_float4(v[0], v[1], v[2], v[3]);
+  } else {
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (j + e < d) base[off + e] = v[e];
+  }
+}
+
+// kTables: the CSR arrays are read from shared memory (they fit) instead of global memory.
+template <bool kTables>
+__global__ void __launch_bounds__(kCsrThreads, 1) step_csr_kernel(const StepParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int n = p.n, S = p.S, pitch = S + kCsrPad, tid = threadIdx.x;
+  double* sx = reinterpret_cast<double*>(smem_raw);
+  double* sy = sx + static_cast<size_t>(n) * pitch;
+  const double* vals = p.vals;
+  const int32_t* rows = p.row_ptr;
+  const int32_t* cols = p.col_idx;
+  if (kTables) {
+    double* s_val = sy + static_cast<size_t>(n) * pitch;
+    int32_t* s_row = reinterpret_cast<int32_t*>(s_val + p.nnz);
+    int32_t* s_col = s_row + (n + 1);
+    for (int k = tid; k < p.nnz; k += kCsrThreads) {
+      s_val[k] = p.vals[k];
+      s_col[k] = p.col_idx[k];
+    }
+    for (int k = tid; k <= n; k += kCsrThreads) s_row[k] = p.row_ptr[k];
+    vals = s_val;
+    rows = s_row;
+    cols = s_col;
+    __syncthreads();  // the tables are read right below
+  }
+  // item = ((row quad * groups + coordinate group) * 4 + row within quad): the four rows of a Philox call in
+  // four neighbouring lanes
+  const int groups = S >> 2;
+  const int r4 = tid & 3, cg = (tid >> 2) % groups, q = (tid >> 2) / groups;
+  const int i = 4 * q + r4;
+  const bool owner = q < (n + 3) / 4 && i < n;  // threads without an element idle (they still meet the barriers)
+  const int k0 = owner ? rows[i] : 0, k1 = owner ? rows[i + 1] : 0;
+  const double one_plus_eta = 1.0 + p.eta, eta = p.eta, alpha = p.alpha;
+  const float sigma = static_cast<float>(p.sigma);
+  const bool dpsgd = p.mode == kModeDpsgd, external = p.mode == kModeExternal;
+  double* my_x = sx + static_cast<size_t>(owner ? i : 0) * pitch + 4 * cg;
+  double* my_y = sy + static_cast<size_t>(owner ? i : 0) * pitch + 4 * cg;
 
   for (long long slab = blockIdx.x; slab < p.num_slabs; slab += gridDim.x) {
-    const long long j0 = slab * S;
-    const int width = static_cast<int>(min(static_cast<long long>(S), p.d - j0));
-    __syncthreads();  // the previous slab's epilogue has finished reading the buffers
-
-    for (int e = tid; e < NS; e += kCsrThreads) {
-      const int i = e >> p.log2S, col = e & (S - 1);
-      double vx = 0.0, vy = 0.0;
-      if (col < width) {
-        const long long off = static_cast<long long>(i) * p.ld + j0 + col;
-        vx = static_cast<double>(p.x[off]);
-        if (p.mode != kModeDpsgd) vy = static_cast<double>(p.y[off]);
-        if (p.mode == kModeExternal)  // Algorithm 2's tracker update with the caller's newest gradient
-          vy += static_cast<double>(p.g_ext[off]) - static_cast<double>(p.g[off]);
+    const long long j = slab * S + 4 * cg;  // this thread's first coordinate
+    const long long off = static_cast<long long>(i) * p.ld + j;
+    const bool active = owner && j < p.d;
+    double px[4], py[4];  // z_{r-1} of this thread's elements; z_r is in the slab
+    float gold[4] = {0.f, 0.f, 0.f, 0.f};
+    if (active) {
+      float xv[4], yv[4] = {0.f, 0.f, 0.f, 0.f};
+      load4(p.x, off, j, p.d, xv);
+      if (!dpsgd) load4(p.y, off, j, p.d, yv);
+      if (external) {  // Algorithm 2's tracker update with the caller's newest gradient
+        float gn[4];
+        load4(p.g_ext, off, j, p.d, gn);
+        load4(p.g, off, j, p.d, gold);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          px[e] = static_cast<double>(xv[e]);
+          py[e] = static_cast<double>(yv[e]) + (static_cast<double>(gn[e]) - static_cast<double>(gold[e]));
+          gold[e] = gn[e];  // what the step stores as the gradient folded last
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          px[e] = static_cast<double>(xv[e]);
+          py[e] = static_cast<double>(yv[e]);
+        }
       }
-      cur_x[e] = vx;
-      prv_x[e] = vx;
-      cur_y[e] = vy;
-      prv_y[e] = vy;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) px[e] = py[e] = 0.0;
+    }
+    __syncthreads();  // the previous slab's rounds have finished reading the slab
+    if (owner) {
+      *reinterpret_cast<double2*>(my_x) = make_double2(px[0], px[1]);
+      *reinterpret_cast<double2*>(my_x + 2) = make_double2(px[2], px[3]);
+      *reinterpret_cast<double2*>(my_y) = make_double2(py[0], py[1]);
+      *reinterpret_cast<double2*>(my_y + 2) = make_double2(py[2], py[3]);
     }
     __syncthreads();
 
-    double *cx = cur_x, *cy = cur_y, *px = prv_x, *py = prv_y;
+    // z_r lives in the slab, z_{r-1} of this thread's elements in px, py; after the loop cx, cy hold z_K
+    double cx[4], cy[4];
     for (int r = 0; r < p.K; ++r) {
-      for (int e = tid; e < NS; e += kCsrThreads) {
-        const int i = e >> p.log2S, col = e & (S - 1);
-        double ax = 0.0, ay = 0.0;
-        const int k_end = s_row[i + 1];
-        for (int k = s_row[i]; k < k_end; ++k) {
-          const double w = s_val[k];
-          const int src = (s_col[k] << p.log2S) + col;
-          ax = fma(w, cx[src], ax);
-          ay = fma(w, cy[src], ay);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) cx[e] = cy[e] = 0.0;
+      for (int k = k0; k < k1; ++k) {
+        const double w = vals[k];
+        const size_t src = static_cast<size_t>(cols[k]) * pitch + 4 * cg;
+        const double2 x01 = *reinterpret_cast<const double2*>(sx + src);
+        const double2 x23 = *reinterpret_cast<const double2*>(sx + src + 2);
+        cx[0] = fma(w, x01.x, cx[0]);
+        cx[1] = fma(w, x01.y, cx[1]);
+        cx[2] = fma(w, x23.x, cx[2]);
+        cx[3] = fma(w, x23.y, cx[3]);
+        if (!dpsgd) {
+          const double2 y01 = *reinterpret_cast<const double2*>(sy + src);
+          const double2 y23 = *reinterpret_cast<const double2*>(sy + src + 2);
+          cy[0] = fma(w, y01.x, cy[0]);
+          cy[1] = fma(w, y01.y, cy[1]);
+          cy[2] = fma(w, y23.x, cy[2]);
+          cy[3] = fma(w, y23.y, cy[3]);
         }
-        px[e] = fma(one_plus_eta, ax, -eta * px[e]);
-        py[e] = fma(one_plus_eta, ay, -eta * py[e]);  // D-PSGD: an all-zero slab, never stored
       }
-      __syncthreads();
-      double* t;
-      t = cx; cx = px; px = t;
-      t = cy; cy = py; py = t;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        cx[e] = fma(one_plus_eta, cx[e], -eta * px[e]);
+        cy[e] = fma(one_plus_eta, cy[e], -eta * py[e]);
+      }
+      if (r + 1 < p.K) {
+        if (owner) {  // this round's own values become the next round's "previous"
+          const double2 x01 = *reinterpret_cast<const double2*>(my_x), x23 = *reinterpret_cast<const double2*>(my_x + 2);
+          px[0] = x01.x; px[1] = x01.y; px[2] = x23.x; px[3] = x23.y;
+          if (!dpsgd) {
+            const double2 y01 = *reinterpret_cast<const double2*>(my_y), y23 = *reinterpret_cast<const double2*>(my_y + 2);
+            py[0] = y01.x; py[1] = y01.y; py[2] = y23.x; py[3] = y23.y;
+          }
+        }
+        __syncthreads();  // everybody has read round r's values
+        if (owner) {
+          *reinterpret_cast<double2*>(my_x) = make_double2(cx[0], cx[1]);
+          *reinterpret_cast<double2*>(my_x + 2) = make_double2(cx[2], cx[3]);
+          if (!dpsgd) {
+            *reinterpret_cast<double2*>(my_y) = make_double2(cy[0], cy[1]);
+            *reinterpret_cast<double2*>(my_y + 2) = make_double2(cy[2], cy[3]);
+          }
+        }
+        __syncthreads();
+      }
     }
 
-    // element-wise tail of the step; a thread takes the four workers 4q..4q+3 of one coordinate
-    for (int it = tid; it < nq * S; it += kCsrThreads) {
-      const int q = it >> p.log2S, col = it & (S - 1);
-      if (col >= width) continue;
-      const long long j = j0 + col;
-      float xi[4] = {0.f, 0.f, 0.f, 0.f};
-      if (sigma != 0.0 && p.mode != kModeExternal)
-        normal_quad(p.seed_lo, p.seed_hi, static_cast<unsigned long long>(p.coord_offset + j), q, p.t_noise, xi);
+    // ---- element-wise tail of the step on the thread's four elements
+    float xi[4] = {0.f, 0.f, 0.f, 0.f};
+    if (sigma != 0.f && !external) {  // every lane takes part (the shuffles want whole warps); idle lanes' draws are unused
+      // lane r4 draws coordinate j + r4 for the quad's four workers; the transpose gives it its own row's four
+      normal_quad(p.seed_lo, p.seed_hi, static_cast<unsigned long long>(p.coord_offset + j + r4), static_cast<uint32_t>(q),
+                  p.t_noise, xi);
+      transpose_rows(xi, r4);
+    }
+    if (active) {
+      float xo[4], yo[4], go[4];
+      if (external) {
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        const int i = 4 * q + w;
-        if (i < n) {
-          const long long off = static_cast<long long>(i) * p.ld + j;
-          if (p.mode == kModeExternal) {
-            const double y_gossip = cy[i * S + col];
-            p.x[off] = static_cast<float>(cx[i * S + col] - alpha * y_gossip);
-            p.y[off] = static_cast<float>(y_gossip);
-            p.g[off] = p.g_ext[off];  // the gradient just folded is the next step's g_old
-            if (p.y_obs != nullptr) p.y_obs[off] = static_cast<float>(y_gossip);
-            continue;
-          }
-          if (p.mode == kModeDpsgd) {
-            const double x_new = cx[i * S + col] - alpha * static_cast<double>(p.g[off]);
-            const float x_new_f = static_cast<float>(x_new);
-            const double g_new = fma(static_cast<double>(p.a[off]), x_new - static_cast<double>(p.c[off]),
-                                     sigma * static_cast<double>(xi[w]));
-            p.x[off] = x_new_f;
-            p.g[off] = static_cast<float>(g_new);
-            continue;
-          }
-          const double y_gossip = cy[i * S + col];
-          const double x_new = cx[i * S + col] - alpha * y_gossip;
-          // gradient point: the new model, or (Algorithm 2 as printed) the model this step started from,
-          // which is still in global memory because this thread overwrites it only below
-          const double x_at = p.grad_at_start ? static_cast<double>(p.x[off]) : x_new;
-          const double g_new = fma(static_cast<double>(p.a[off]), x_at - static_cast<double>(p.c[off]),
-                                   sigma * static_cast<double>(xi[w]));
-          const float g_new_f = static_cast<float>(g_new);
-          const double y_new = y_gossip + (static_cast<double>(g_new_f) - static_cast<double>(p.g[off]));
-          p.x[off] = static_cast<float>(x_new);
-          p.y[off] = static_cast<float>(y_new);
-          p.g[off] = g_new_f;
-          if (p.y_obs != nullptr) p.y_obs[off] = static_cast<float>(y_gossip);
+        for (int e = 0; e < 4; ++e) {
+          xo[e] = static_cast<float>(cx[e] - alpha * cy[e]);
+          yo[e] = static_cast<float>(cy[e]);  // the gossiped tracker
+          go[e] = gold[e];                    // the gradient just folded is the next step's g_old
         }
+      } else {
+        float av[4], cv[4], gv[4], xold[4];
+        load4(p.a, off, j, p.d, av);
+        load4(p.c, off, j, p.d, cv);
+        load4(p.g, off, j, p.d, gv);
+        if (p.grad_at_start) load4(p.x, off, j, p.d, xold);  // still the old model: this thread overwrites it below
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const double x_new = dpsgd ? cx[e] - alpha * static_cast<double>(gv[e]) : cx[e] - alpha * cy[e];
+          // gradient point: the new model, or (Algorithm 2 as printed) the model this step started from
+          const double x_at = p.grad_at_start ? static_cast<double>(xold[e]) : x_new;
+          const double g_new = fma(static_cast<double>(av[e]), x_at - static_cast<double>(cv[e]),
+                                   static_cast<double>(sigma) * static_cast<double>(xi[e]));
+          go[e] = static_cast<float>(g_new);
+          xo[e] = static_cast<float>(x_new);
+          yo[e] = static_cast<float>(cy[e] + (static_cast<double>(go[e]) - static_cast<double>(gv[e])));
+        }
+      }
+      store4(p.x, off, j, p.d, xo);
+      if (!dpsgd) store4(p.y, off, j, p.d, yo);
+      store4(p.g, off, j, p.d, go);
+      if (p.y_obs != nullptr && !dpsgd) {
+        float yg[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) yg[e] = static_cast<float>(cy[e]);
+        store4(p.y_obs, off, j, p.d, yg);
       }
     }
   }
@@ -147,38 +247,34 @@ __global__ void __launch_bounds__(kCsrThreads) step_csr_kernel(const StepParams 
 
 }  // namespace
 
+// Chooses the slab width: the widest power of two (4 .. 64 coordinates) for which every (worker quad, four
+// coordinates) item has a thread of its own and the slabs fit; the CSR arrays join them in shared memory if there
+// is room.  p.log2S < 0 afterwards means the tables stay in global memory.
 int plan_step_csr(StepParams& p, int smem_optin_bytes) {
-  // Largest power-of-two slab (<= 128 coordinates) whose buffers leave room for two CTAs per SM;
-  // fall back to one CTA per SM with the widest slab that fits at all.
-  const size_t two_cta_budget = 110 * 1024;
+  const int quads = (p.n + 3) / 4;
   int best = 0;
-  for (int S = 128; S >= 4; S >>= 1)
-    if (csr_smem_bytes(p.n, p.nnz, S) <= two_cta_budget) { best = S; break; }
-  if (best < 16) {
-    for (int S = 16; S >= 4; S >>= 1)
-      if (csr_smem_bytes(p.n, p.nnz, S) <= static_cast<size_t>(smem_optin_bytes)) { best = S; break; }
+  for (int S = 64; S >= 4; S >>= 1) {
+    if (quads * 4 * (S / 4) > kCsrThreads) continue;
+    if (csr_smem_bytes(p.n, p.nnz, S, false) > static_cast<size_t>(smem_optin_bytes)) continue;
+    best = S;
+    break;
   }
   if (best == 0) return DETAG_ERR_UNSUPPORTED;
   p.S = best;
-  p.log2S = 0;
-  while ((1 << p.log2S) < best) ++p.log2S;
+  p.log2S = csr_smem_bytes(p.n, p.nnz, best, true) <= static_cast<size_t>(smem_optin_bytes) ? 1 : -1;
   p.num_slabs = (p.d + best - 1) / best;
   return DETAG_OK;
 }
 
 int launch_step_csr(const StepParams& p, int sm_count, cudaStream_t stream) {
-  const size_t smem = csr_smem_bytes(p.n, p.nnz, p.S);
-  const int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(step_csr_kernel), static_cast<int>(smem));
+  const bool tables = p.log2S > 0;
+  const size_t smem = csr_smem_bytes(p.n, p.nnz, p.S, tables);
+  auto kernel = tables ? step_csr_kernel<true> : step_csr_kernel<false>;
+  const int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), static_cast<int>(smem));
   if (rc != 0) return rc;
-  int per_sm = 1;
-  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, step_csr_kernel, kCsrThreads, smem);
-  if (e != cudaSuccess) return static_cast<int>(e);
-  if (per_sm < 1) per_sm = 1;
-  const long long grid = p.num_slabs < static_cast<long long>(sm_count) * per_sm
-                             ? p.num_slabs
-                             : static_cast<long long>(sm_count) * per_sm;
+  const long long grid = p.num_slabs < static_cast<long long>(sm_count) ? p.num_slabs : static_cast<long long>(sm_count);
   if (grid <= 0) return 0;
-  step_csr_kernel<<<static_cast<unsigned>(grid), kCsrThreads, smem, stream>>>(p);
+  kernel<<<static_cast<unsigned>(grid), kCsrThreads, smem, stream>>>(p);
   return static_cast<int>(cudaGetLastError());
 }
 
