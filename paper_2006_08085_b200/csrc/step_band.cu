@@ -33,8 +33,7 @@ namespace detag {
 namespace {
 
 constexpr int kR = 32;             // output rows per tile
-constexpr int kHalo = 16;          // window rows on each side = largest supported half-band
-constexpr int kW = kR + 2 * kHalo; // window rows
+constexpr int kW = 64;             // window rows: all (padded) workers
 constexpr int kS = 64;             // coordinates per tile: 8 MMA tiles of 8, one per consumer warp of a group
 constexpr int kPitchXY = kS + 8;   // floats; 8 mod 32 -> the four window rows of a B fragment hit disjoint banks
 constexpr int kPitchE = kS + 8;    // floats; rows of g, a, c: consecutive rows 8t + r of the accumulator layout
@@ -47,10 +46,9 @@ constexpr int kGroupWarps = kS / 8;
 constexpr int kConsumerWarps = kGroupWarps * kWarpGroups;
 constexpr int kProducerWarp = kConsumerWarps, kStoreWarp = kConsumerWarps + 1, kSignalWarp = kConsumerWarps + 2;
 constexpr int kThreads = (kConsumerWarps + 3) * 32;
-constexpr int kSideFloats = 2 * kHalo * kPitchXY;  // rows 0..15 of x and y, kept for the slab's last row block
 constexpr int kOutFloats = 3 * kR * kS;
 constexpr size_t kSmemBytes =
-    static_cast<size_t>(kStages) * kStageBytes + 2 * kSideFloats * 4 + kWarpGroups * kOutFloats * 4 + 128;  // + barriers, counters
+    static_cast<size_t>(kStages) * kStageBytes + kWarpGroups * kOutFloats * 4 + 128;  // + barriers, counters
 constexpr int kDenseFragBytes = 2 * (kW / 4) * 4 * 32 * 8;  // dense mode: [row block][window step][t][lane] doubles
 static_assert(kSmemBytes + kDenseFragBytes <= 232448, "shared memory plan");
 
@@ -78,12 +76,10 @@ __device__ __forceinline__ void transpose4(float (&v)[4], int q) {
 
 __global__ void __launch_bounds__(kThreads, 1)
 step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps) {
-  constexpr bool kDense = true;  // the whole 64-row window, every block of P
   // No static shared memory: the dynamic array starts at the CTA's shared window; its alignment is checked.
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* stage_mem = reinterpret_cast<float*>(smem_raw);
-  float* side_mem = stage_mem + kStages * kStageFloats;  // [slab parity][x, y][16][kPitchXY]
-  float* out_mem = side_mem + 2 * kSideFloats;           // [group][x', y', g'][32][kS]
+  float* out_mem = stage_mem + kStages * kStageFloats;   // [group][x', y', g'][32][kS]
   uint64_t* full = reinterpret_cast<uint64_t*>(out_mem + kWarpGroups * kOutFloats);
   uint64_t* empty = full + kStages;
   uint64_t* out_ready = empty + kStages;
@@ -93,12 +89,12 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps) {
   double* frag = reinterpret_cast<double*>(smem_raw + kSmemBytes);  // dense mode only (the launch adds the bytes)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = p.n;
-  const int row_blocks = kDense ? 2 : n / kR;
+  constexpr int row_blocks = 2;  // 64 padded rows
   if ((s_addr(smem_raw) & 127u) != 0) {
     if (tid == 0) atomicExch(p.status, 2);
     return;
   }
-  if (kDense) {
+  {
     // slice rb of P in fragment order: block (ws, t), lane (r, kq) holds P[32 rb + 8t + r][4 ws + kq]
     for (int e = tid; e < 2 * (kW / 4) * 4 * 32; e += kThreads) {
       const int l = e & 31, t = (e >> 5) & 3, ws = (e >> 7) % (kW / 4), b = e / (32 * 4 * (kW / 4));
@@ -156,24 +152,12 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps) {
         const long long slab = blockIdx.x + slab_no * gridDim.x;
         float* st = stage_mem + static_cast<size_t>(s) * kStageFloats;
         const int col = static_cast<int>(slab * kS);
-        const bool last = !kDense && rb == row_blocks - 1;
-        // the last block's final window piece (rows 0..15) is not loaded: it comes from the side buffer
-        const unsigned bytes = static_cast<unsigned>(kStageBytes) - (last ? 2u * 16 * kPitchXY * 4 : 0u) +
-                               (!kDense && rb == 0 ? static_cast<unsigned>(kSideFloats) * 4 : 0u);
-        bar_expect_tx(&full[s], bytes);
+        bar_expect_tx(&full[s], static_cast<unsigned>(kStageBytes));
 #pragma unroll
-        for (int q = 0; q < kW / 16; ++q) {  // the window wraps around the ring in 16-row pieces
-          if (last && q == kW / 16 - 1) continue;
-          const int row = kDense ? 16 * q : ((rb * kR - kHalo + 16 * q) % n + n) % n;
+        for (int q = 0; q < kW / 16; ++q) {  // the window = all 64 rows, in 16-row pieces
+          const int row = 16 * q;
           tile_load(st + q * 16 * kPitchXY, &maps.x16, col, row, &full[s]);
           tile_load(st + kW * kPitchXY + q * 16 * kPitchXY, &maps.y16, col, row, &full[s]);
-        }
-        if (!kDense && rb == 0) {
-          // Rows 0..15 before anything of this slab is stored.  The buffer of this parity was last read by the
-          // last block of the slab before the previous one, whose stage has been recycled since.
-          float* sd = side_mem + static_cast<size_t>(slab_no & 1) * kSideFloats;
-          tile_load(sd, &maps.x16, col, 0, &full[s]);
-          tile_load(sd + kHalo * kPitchXY, &maps.y16, col, 0, &full[s]);
         }
         float* se = st + 2 * kW * kPitchXY;
 #pragma unroll
@@ -263,11 +247,6 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps) {
     const float* sg = sy + kW * kPitchXY;
     const float* sa = sg + kR * kPitchE;
     const float* sc = sa + kR * kPitchE;
-    // window rows 48..63 of the slab's last block are rows 0..15 of the ring: kept in the side buffer
-    const bool wrap_side = !kDense && rb == row_blocks - 1;
-    // offsets (in floats, relative to sx / sy) that redirect window rows 48..63 to the side buffer
-    const int side_dx = static_cast<int>(side_mem + (slab_no & 1) * kSideFloats - sx) - (kW - kHalo) * kPitchXY;
-    const int side_dy = side_dx + kHalo * kPitchXY - kW * kPitchXY;
     const long long j0 = slab * kS;
     const long long j = j0 + cl + 2 * kq;
     const bool active = j0 + cl < p.d;  // a tile wholly beyond column d computes nothing but keeps the protocol
@@ -287,9 +266,8 @@ step_band_kernel(const StepParams p, const __grid_constant__ BandMaps maps) {
 #pragma unroll
       for (int ws = 0; ws < kW / 4; ++ws) {  // window steps of four rows
         const int src = (4 * ws + kq) * kPitchXY + cl + r;
-        const bool side = ws >= (kW - kHalo) / 4 && wrap_side;
-        const double by = static_cast<double>(sy[src + (side ? side_dy : 0)]);
-        const double bx = fma(-alpha, by, static_cast<double>(sx[src + (side ? side_dx : 0)]));
+        const double by = static_cast<double>(sy[src]);
+        const double bx = fma(-alpha, by, static_cast<double>(sx[src]));
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
           const double a = frag[((rb * (kW / 4) + ws) * 4 + t) * 32 + lane];
