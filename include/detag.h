@@ -57,12 +57,16 @@ enum {
 /* Kernel variants of the gossip part of the step; all compute the same result. */
 enum {
   DETAG_VARIANT_AUTO = 0,  /* host cost model picks */
-  DETAG_VARIANT_CSR = 1,   /* K rounds of neighbour-indexed sums over the CSR rows, slab staged on chip */
+  DETAG_VARIANT_CSR = 1,   /* K rounds of neighbour-indexed sums over the CSR rows, slab staged on chip: any graph, n <= 1024 */
   DETAG_VARIANT_DENSE = 2, /* one product with the host-precomputed polynomial P_K(M), n <= 64 */
-  DETAG_VARIANT_RING = 3,  /* banded circulant polynomial P_K(M): circulant M (rings), n % 32 == 0, n >= 64, K*bandwidth <= 16 */
+  DETAG_VARIANT_RING = 3,  /* circulant M (rings), n % 32 == 0, 64 <= n <= 1024: the circulant polynomial P_K(M) as a band
+                              while K * bandwidth <= 16, as a dense circulant (n <= 256) beyond, e.g. at Theorem 3's phase
+                              length; the last d % 64 coordinates run through the CSR kernel in the same call */
   DETAG_VARIANT_TORUS = 4  /* block-circulant M with 8-worker blocks, symmetric in the block distance (R x 8 tori, n = 32 or 64):
                               Fourier transform along the block axis, one 8 x 8 polynomial block per frequency, transform back */
 };
+/* Caller-written gradients run on DENSE (n <= 32) and CSR, D-PSGD on DENSE (n <= 32), RING and CSR; AUTO picks among
+   those, a forced variant outside them makes detag_step return DETAG_ERR_UNSUPPORTED. */
 
 /* The point at which a step queries the stochastic gradient oracle. */
 enum {
