@@ -17,7 +17,7 @@ namespace {
 size_t align_up(size_t v) { return (v + detag::kWsAlign - 1) / detag::kWsAlign * detag::kWsAlign; }
 
 struct WsLayout {
-  size_t status, result, row_ptr, col_idx, vals, poly, torus, circ_row, partials, total;
+  size_t status, result, row_ptr, col_idx, vals, poly, torus, circ_row, wide, partials, total;
 };
 
 WsLayout ws_layout(const detag_state* s) {
@@ -38,6 +38,8 @@ WsLayout ws_layout(const detag_state* s) {
   off += align_up(s->torus_frag.size() * sizeof(double));
   l.circ_row = off;
   off += align_up(s->circ_row.size() * sizeof(double));
+  l.wide = off;
+  off += align_up(s->wide_frag.size() * sizeof(double));
   l.partials = off;
   off += align_up(detag::kMaxPartials * sizeof(double));
   l.total = off;
@@ -229,6 +231,7 @@ StepParams make_params(const detag_state* s) {
   p.poly = s->d_poly;
   p.torus = s->d_torus;
   p.circ_row = s->d_circ_row;
+  p.wide = s->d_wide;
   p.eta = s->eta;
   p.alpha = s->alpha;
   p.sigma = s->sigma;
@@ -244,7 +247,9 @@ StepParams make_params(const detag_state* s) {
 }
 
 bool dense_ok(const detag_state* s) {
-  return !s->poly.empty() && s->d <= 0x7fffffffLL && detag::dense_variant_available(s->n);
+  if (s->d > 0x7fffffffLL) return false;
+  return (!s->poly.empty() && detag::dense_variant_available(s->n)) ||
+         (!s->wide_frag.empty() && detag::wide_variant_available(s->n));
 }
 
 // Host cost model.  The dense product needs n multiply-adds per element and array against the sparse
@@ -257,7 +262,7 @@ bool dense_ok(const detag_state* s) {
 bool variant_runs_mode(const detag_state* s, int variant) {
   if (step_mode(s) == detag::kModeDetag) return true;
   if (variant == DETAG_VARIANT_RING) return step_mode(s) == detag::kModeDpsgd;
-  return variant == DETAG_VARIANT_CSR || (variant == DETAG_VARIANT_DENSE && s->n <= 32);
+  return variant == DETAG_VARIANT_CSR || (variant == DETAG_VARIANT_DENSE && s->n <= 32);  // n > 32: DeTAG step only
 }
 
 int resolve_variant(const detag_state* s) {
@@ -286,7 +291,7 @@ int query_device(detag_state* s) {
 }
 
 // Kernel families that take tensor maps.
-enum { kFamilyMma = 1, kFamilyBand = 2, kFamilyTorus = 3, kFamilyRing = 4 };
+enum { kFamilyMma = 1, kFamilyBand = 2, kFamilyTorus = 3, kFamilyRing = 4, kFamilyWide = 5 };
 
 // Tensor maps for the buffers in `p`: built on first use, then found again by buffer addresses and sizes
 // (detag_step always hits; detag_step_host cycles through its two chunk slots and the ragged last chunk).
@@ -312,6 +317,7 @@ const detag::TensorMapSet* maps_for(detag_state* s, int family, const StepParams
   const bool ok = family == kFamilyMma    ? detag::build_maps_mma(p, &en.maps)
                   : family == kFamilyBand ? detag::build_maps_band(p, &en.maps)
                   : family == kFamilyRing ? detag::build_maps_ring(p, &en.maps)
+                  : family == kFamilyWide ? detag::build_maps_wide(p, &en.maps)
                                           : detag::build_maps_torus(p, &en.maps);
   if (!ok) return nullptr;
   en.family = family;
@@ -319,6 +325,24 @@ const detag::TensorMapSet* maps_for(detag_state* s, int family, const StepParams
   en.ld = p.ld;
   std::memcpy(en.ptr, key, sizeof key);
   return &en.maps;
+}
+
+// The columns from `first` on through the generic rounds kernel (the tensor-path kernels that take whole 32- or
+// 64-coordinate pieces hand their remainder here, in the same call).
+int launch_tail_columns(detag_state* s, const StepParams& p, long long first, cudaStream_t stream, int* cuda_error) {
+  StepParams pt = p;
+  pt.d = p.d - first;
+  pt.coord_offset = p.coord_offset + first;
+  pt.x = p.x + first;
+  pt.y = p.y + first;
+  pt.g = p.g + first;
+  pt.a = p.a + first;
+  pt.c = p.c + first;
+  if (p.y_obs) pt.y_obs = p.y_obs + first;
+  const int rc = detag::plan_step_csr(pt, s->smem_optin);
+  if (rc != DETAG_OK) return fail(s, rc, "graph too large for the shared-memory plan");
+  *cuda_error = detag::launch_step_csr(pt, s->sm_count, stream);
+  return DETAG_OK;
 }
 
 // Picks the kernel variant, plans it for the sizes in `p` and launches it.
@@ -334,6 +358,23 @@ int launch_step(detag_state* s, StepParams& p, cudaStream_t stream) {
     return fail(s, DETAG_ERR_UNBOUND, "caller-written gradients selected but no gradient array given");
   switch (variant) {
     case DETAG_VARIANT_DENSE: {
+      if (p.n > detag::kMaxDenseWorkers) {
+        // the register-resident polynomial takes whole 32-coordinate halves; the last d % 32 columns go to the generic kernel
+        const long long d_main = p.d & ~31LL;
+        if (d_main > 0) {
+          StepParams pm = p;
+          pm.d = d_main;
+          const detag::TensorMapSet* maps = maps_for(s, kFamilyWide, pm);
+          if (!maps) return fail(s, DETAG_ERR_CUDA, "tensor map encoding failed");
+          e = detag::launch_step_wide(pm, *maps, p.wide, s->sm_count, stream);
+          if (e != 0) return fail_cuda(s, e, "step kernel launch");
+        }
+        if (d_main < p.d) {
+          const int rc = launch_tail_columns(s, p, d_main, stream, &e);
+          if (rc != DETAG_OK) return rc;
+        }
+        break;
+      }
       const bool mma = p.n <= 32;
       const detag::TensorMapSet* maps = maps_for(s, mma ? kFamilyMma : kFamilyBand, p);
       if (!maps) return fail(s, DETAG_ERR_CUDA, "tensor map encoding failed");
@@ -353,18 +394,8 @@ int launch_step(detag_state* s, StepParams& p, cudaStream_t stream) {
         if (e != 0) return fail_cuda(s, e, "step kernel launch");
       }
       if (d_main < p.d) {
-        StepParams pt = p;
-        pt.d = p.d - d_main;
-        pt.coord_offset = p.coord_offset + d_main;
-        pt.x = p.x + d_main;
-        pt.y = p.y + d_main;
-        pt.g = p.g + d_main;
-        pt.a = p.a + d_main;
-        pt.c = p.c + d_main;
-        if (p.y_obs) pt.y_obs = p.y_obs + d_main;
-        const int rc = detag::plan_step_csr(pt, s->smem_optin);
-        if (rc != DETAG_OK) return fail(s, rc, "graph too large for the shared-memory plan");
-        e = detag::launch_step_csr(pt, s->sm_count, stream);
+        const int rc = launch_tail_columns(s, p, d_main, stream, &e);
+        if (rc != DETAG_OK) return rc;
       }
       break;
     }
@@ -429,7 +460,13 @@ int detag_create(detag_state** out, int n, int64_t d, const int32_t* row_ptr, co
   s->row_ptr.assign(row_ptr, row_ptr + n + 1);
   s->col_idx.assign(col_idx, col_idx + nnz);
   s->vals.assign(vals, vals + nnz);
-  if (n <= detag::kMaxDenseWorkers) gossip_polynomial(s, s->poly);
+  if (n <= detag::kMaxDenseWorkers) {
+    gossip_polynomial(s, s->poly);
+  } else if (n <= detag::kMaxWideWorkers) {  // kept as the warp strips of the register-resident kernel only
+    std::vector<double> poly;
+    gossip_polynomial(s, poly);
+    detag::wide_fragments(n, poly, s->wide_frag);
+  }
   analyse_circulant(s);
   analyse_torus(s);
   s->map_cache.reserve(8);
@@ -468,6 +505,7 @@ int detag_bind(detag_state* s, int64_t ld, float* x, float* y, float* g, const f
   s->d_poly = s->poly.empty() ? nullptr : reinterpret_cast<double*>(base + l.poly);
   s->d_torus = s->torus_frag.empty() ? nullptr : reinterpret_cast<double*>(base + l.torus);
   s->d_circ_row = s->circ_row.empty() ? nullptr : reinterpret_cast<double*>(base + l.circ_row);
+  s->d_wide = s->wide_frag.empty() ? nullptr : reinterpret_cast<double*>(base + l.wide);
   s->d_partials = reinterpret_cast<double*>(base + l.partials);
 
   e = cudaMemset(base, 0, detag::kWsAlign);
@@ -483,6 +521,8 @@ int detag_bind(detag_state* s, int64_t ld, float* x, float* y, float* g, const f
     e = cudaMemcpy(s->d_torus, s->torus_frag.data(), s->torus_frag.size() * sizeof(double), cudaMemcpyHostToDevice);
   if (e == cudaSuccess && s->d_circ_row)
     e = cudaMemcpy(s->d_circ_row, s->circ_row.data(), s->circ_row.size() * sizeof(double), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess && s->d_wide)
+    e = cudaMemcpy(s->d_wide, s->wide_frag.data(), s->wide_frag.size() * sizeof(double), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) return fail_cuda(s, e, "detag_bind: workspace upload");
 
   s->ld = ld;
@@ -521,7 +561,7 @@ int detag_set_variant(detag_state* s, int variant) {
     case DETAG_VARIANT_CSR:
       break;
     case DETAG_VARIANT_DENSE:
-      if (!dense_ok(s)) return fail(s, DETAG_ERR_UNSUPPORTED, "detag_set_variant: dense variant needs n <= 64");
+      if (!dense_ok(s)) return fail(s, DETAG_ERR_UNSUPPORTED, "detag_set_variant: dense variant needs n <= 128");
       break;
     case DETAG_VARIANT_TORUS:
       if (!torus_ok(s))
@@ -747,6 +787,9 @@ int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* 
   if (e == cudaSuccess && !s->circ_row.empty())
     e = cudaMemcpyAsync(base + l.circ_row, s->circ_row.data(), s->circ_row.size() * sizeof(double),
                         cudaMemcpyHostToDevice, user);
+  if (e == cudaSuccess && !s->wide_frag.empty())
+    e = cudaMemcpyAsync(base + l.wide, s->wide_frag.data(), s->wide_frag.size() * sizeof(double), cudaMemcpyHostToDevice,
+                        user);
   if (e == cudaSuccess) e = cudaEventRecord(s->host_event[2], user);
   for (int k = 0; k < 2 && e == cudaSuccess; ++k) e = cudaStreamWaitEvent(s->host_stream[k], s->host_event[2], 0);
   if (e != cudaSuccess) return fail_cuda(s, e, "detag_step_host: table upload");
@@ -758,6 +801,7 @@ int detag_step_host(detag_state* s, int64_t ld_host, float* x, float* y, float* 
   p.poly = s->poly.empty() ? nullptr : reinterpret_cast<double*>(base + l.poly);
   p.torus = s->torus_frag.empty() ? nullptr : reinterpret_cast<double*>(base + l.torus);
   p.circ_row = s->circ_row.empty() ? nullptr : reinterpret_cast<double*>(base + l.circ_row);
+  p.wide = s->wide_frag.empty() ? nullptr : reinterpret_cast<double*>(base + l.wide);
   p.status = status_word;
   p.y_obs = nullptr;
   p.t_noise = static_cast<uint32_t>(s->t + 1);

@@ -14,7 +14,8 @@ typedef struct CUstream_st* cudaStream_t;
 namespace detag {
 
 constexpr int kMaxWorkers = 1024;       // detag_create limit on n
-constexpr int kMaxDenseWorkers = 64;    // dense-polynomial variant limit on n
+constexpr int kMaxDenseWorkers = 64;    // dense-polynomial kernels with P in shared memory: limit on n
+constexpr int kMaxWideWorkers = 128;    // dense-polynomial kernel with P in registers: limit on n
 constexpr int kMaxPartials = 2048;      // per-CTA partial sums of the consensus-error reduction
 constexpr size_t kWsAlign = 256;
 
@@ -40,6 +41,7 @@ struct StepParams {
   const double* vals;
   const double* poly;  // dense P_K(M), row-major n x n (null when n > kMaxDenseWorkers)
   const double* circ_row;  // circulant kernel, dense mode: the first row of P_K(M) (or null)
+  const double* wide;  // register-resident dense kernel (64 < n <= 128): the warp strips of P_K(M) in fragment order (or null)
   const double* torus; // block-circulant kernel: per-frequency 8 x 8 polynomial blocks in fragment order (or null)
   double eta;
   double alpha;
@@ -97,6 +99,12 @@ bool torus_variant_available(int n);               // block-circulant kernel: n 
 bool build_maps_torus(const StepParams& p, TensorMapSet* maps);
 int launch_step_torus(StepParams p, const TensorMapSet& maps, const double* phat_frag /* device */, int sm_count,
                       cudaStream_t stream);
+// dense polynomial held in registers (step_wide.cu): 64 < n <= 128, p.d a multiple of 32, DeTAG step only
+bool wide_variant_available(int n);
+void wide_fragments(int n, const std::vector<double>& poly, std::vector<double>& frag);
+bool build_maps_wide(const StepParams& p, TensorMapSet* maps);
+int launch_step_wide(StepParams p, const TensorMapSet& maps, const double* p_frag /* device */, int sm_count,
+                     cudaStream_t stream);
 int launch_consensus_error(const StepParams& p, double* partials, double* result, int sm_count, cudaStream_t stream);
 int launch_init_external(const StepParams& p, int sm_count, cudaStream_t stream);  // y = g = g_ext
 int launch_expire_wait(int* status, unsigned polls, cudaStream_t stream);          // a wait nobody ends (self test)
@@ -121,6 +129,7 @@ struct detag_state {
   // 8 x 8 polynomial blocks in MMA fragment order
   bool torus = false;
   std::vector<double> torus_frag;
+  std::vector<double> wide_frag;  // 64 < n <= 128: P_K(M) as the warp strips of the register-resident kernel
   int variant_forced = DETAG_VARIANT_AUTO;
   int gradient_point = DETAG_GRADIENT_AT_NEW_MODEL;
   int algorithm = DETAG_ALGORITHM_DETAG;
@@ -145,6 +154,7 @@ struct detag_state {
   double* d_poly = nullptr;
   double* d_torus = nullptr;
   double* d_circ_row = nullptr;
+  double* d_wide = nullptr;
   double* d_partials = nullptr;
 
   double sigma = 0.0;

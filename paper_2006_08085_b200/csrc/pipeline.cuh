@@ -1,5 +1,5 @@
 // Device-side building blocks shared by the tensor-path step kernels: bounded mbarrier and counter waits,
-// 2-D TMA tile loads and stores, the float64 warp-level multiply-accumulate.
+// TMA tile loads and stores, the float64 warp-level multiply-accumulate, a 4 x 4 transpose over lanes.
 //
 // Every wait is bounded by a poll limit that the launch passes in (StepParams::spin_limit): a wait that runs out
 // returns false, the caller sets the status word and winds down.  Nothing here traps or spins without a limit.
@@ -134,6 +134,23 @@ __device__ __forceinline__ void tile_store(const CUtensorMap* map, int col, int 
                : "memory");
 }
 
+// Box {32 coordinates, 2 halves, box rows} at (half, row) of a three-dimensional map (make_half_map) -> tile
+// [row][half][32] in shared memory, 16-byte chunks swizzled within each 1 KiB; and the store of such a tile.
+__device__ __forceinline__ void rows_load(float* dst, const CUtensorMap* map, int half, int row, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+          s_addr(dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(half), "r"(row), "r"(s_addr(bar))
+      : "memory");
+}
+
+__device__ __forceinline__ void rows_store(const CUtensorMap* map, int half, int row, const float* src) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
+                   reinterpret_cast<uint64_t>(map)),
+               "r"(0), "r"(half), "r"(row), "r"(s_addr(src))
+               : "memory");
+}
+
 __device__ __forceinline__ void store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // The committed stores have finished READING shared memory (the tile may be overwritten).
 __device__ __forceinline__ void store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
@@ -147,6 +164,20 @@ __device__ __forceinline__ void dmma(double (&c)[2], double a, double b) {
   asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
                : "+d"(c[0]), "+d"(c[1])
                : "d"(a), "d"(b));
+}
+
+// 4 x 4 transpose over four neighbouring lanes (lane bits 0 and 1): lane kq gives row kq = v[0..3] and receives
+// column kq.
+__device__ __forceinline__ void transpose_quad(float (&v)[4], int kq) {
+  const bool b0 = (kq & 1) != 0, b1 = (kq & 2) != 0;
+  float s0 = b0 ? v[0] : v[1], s1 = b0 ? v[2] : v[3];
+  float r0 = __shfl_xor_sync(0xffffffffu, s0, 1), r1 = __shfl_xor_sync(0xffffffffu, s1, 1);
+  if (b0) { v[0] = r0; v[2] = r1; } else { v[1] = r0; v[3] = r1; }
+  s0 = b1 ? v[0] : v[2];
+  s1 = b1 ? v[1] : v[3];
+  r0 = __shfl_xor_sync(0xffffffffu, s0, 2);
+  r1 = __shfl_xor_sync(0xffffffffu, s1, 2);
+  if (b1) { v[0] = r0; v[1] = r1; } else { v[2] = r0; v[3] = r1; }
 }
 
 }  // namespace

@@ -87,49 +87,6 @@ struct RingCoef {
   double p[2 * kRHalo + 1];  // band mode: p[delta + 16] = P[i][(i + delta) mod n]
 };
 
-// View of an [n][ld] array as {32 coordinates, d / 32 halves at a stride of 128 bytes, n rows}: a box of two halves
-// is a slab of 64 coordinates whose rows are contiguous 256-byte pieces.  d must be a multiple of 64.
-inline bool make_ring_map(CUtensorMap* m, const float* base, int n, long long d, long long ld, int box_rows) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(kRHalf), static_cast<cuuint64_t>(d / kRHalf), static_cast<cuuint64_t>(n)};
-  const cuuint64_t strides[2] = {kRHalf * sizeof(float), static_cast<cuuint64_t>(ld) * sizeof(float)};
-  const cuuint32_t box[3] = {static_cast<cuuint32_t>(kRHalf), 2, static_cast<cuuint32_t>(box_rows)};
-  const cuuint32_t elem[3] = {1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, elem,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-__device__ __forceinline__ void rows_load(float* dst, const CUtensorMap* map, int half, int row, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
-          s_addr(dst)),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(half), "r"(row), "r"(s_addr(bar))
-      : "memory");
-}
-
-__device__ __forceinline__ void rows_store(const CUtensorMap* map, int half, int row, const float* src) {
-  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
-                   reinterpret_cast<uint64_t>(map)),
-               "r"(0), "r"(half), "r"(row), "r"(s_addr(src))
-               : "memory");
-}
-
-// 4 x 4 transpose over the four lanes that share a coordinate (lane bits 0 and 1): lane kq gives row kq = v[0..3]
-// and receives column kq.
-__device__ __forceinline__ void transpose_over_kq(float (&v)[4], int kq) {
-  const bool b0 = (kq & 1) != 0, b1 = (kq & 2) != 0;
-  float s0 = b0 ? v[0] : v[1], s1 = b0 ? v[2] : v[3];
-  float r0 = __shfl_xor_sync(0xffffffffu, s0, 1), r1 = __shfl_xor_sync(0xffffffffu, s1, 1);
-  if (b0) { v[0] = r0; v[2] = r1; } else { v[1] = r0; v[3] = r1; }
-  s0 = b1 ? v[0] : v[2];
-  s1 = b1 ? v[1] : v[3];
-  r0 = __shfl_xor_sync(0xffffffffu, s0, 2);
-  r1 = __shfl_xor_sync(0xffffffffu, s1, 2);
-  if (b1) { v[0] = r0; v[1] = r1; } else { v[2] = r0; v[3] = r1; }
-}
-
 template <bool kDense>
 __global__ void __launch_bounds__(kRThreads, 1)
 step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, const __grid_constant__ RingCoef coef,
@@ -369,7 +326,7 @@ step_ring_kernel(const StepParams p, const __grid_constant__ RingMaps maps, cons
       for (int hq = 0; hq < 2; ++hq) {
         float v[4];
         normal_quad(p.seed_lo, p.seed_hi, jn, static_cast<uint32_t>(8 * b + 4 * hq + kq), p.t_noise, v);
-        transpose_over_kq(v, kq);  // v[i]: position kq of quad 8 b + 4 hq + i
+        transpose_quad(v, kq);  // v[i]: position kq of quad 8 b + 4 hq + i
 #pragma unroll
         for (int i = 0; i < 4; ++i) xi[4 * hq + i] = v[i];
       }
@@ -517,10 +474,10 @@ bool ring_dense_available(int n) { return n % kRT == 0 && n >= 64 && n <= 256 &&
 bool build_maps_ring(const StepParams& p, TensorMapSet* out) {
   RingMaps& m = *reinterpret_cast<RingMaps*>(out->bytes);
   const float* y = p.mode == kModeDpsgd ? p.x : p.y;  // D-PSGD has no tracker: those maps are never used
-  return make_ring_map(&m.x, p.x, p.n, p.d, p.ld, kChunkRows) && make_ring_map(&m.y, y, p.n, p.d, p.ld, kChunkRows) &&
-         make_ring_map(&m.g, p.g, p.n, p.d, p.ld, kRT) && make_ring_map(&m.a, p.a, p.n, p.d, p.ld, kRT) &&
-         make_ring_map(&m.c, p.c, p.n, p.d, p.ld, kRT) && make_ring_map(&m.xs, p.x, p.n, p.d, p.ld, kRT) &&
-         make_ring_map(&m.ys, y, p.n, p.d, p.ld, kRT);
+  return make_half_map(&m.x, p.x, p.n, p.d, p.ld, kChunkRows) && make_half_map(&m.y, y, p.n, p.d, p.ld, kChunkRows) &&
+         make_half_map(&m.g, p.g, p.n, p.d, p.ld, kRT) && make_half_map(&m.a, p.a, p.n, p.d, p.ld, kRT) &&
+         make_half_map(&m.c, p.c, p.n, p.d, p.ld, kRT) && make_half_map(&m.xs, p.x, p.n, p.d, p.ld, kRT) &&
+         make_half_map(&m.ys, y, p.n, p.d, p.ld, kRT);
 }
 
 // band != nullptr: band mode, the 33 entries p(delta) at index delta + 16.  band == nullptr: dense mode, p_row is a

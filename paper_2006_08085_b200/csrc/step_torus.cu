@@ -79,51 +79,6 @@ struct TorusMaps {
 };
 static_assert(sizeof(TorusMaps) <= sizeof(TensorMapSet), "tensor map storage");
 
-// View of an [n][ld] array as {32 coordinates, d / 32 halves at a stride of 128 bytes, n rows}: a box of two halves
-// is a slab of 64 coordinates whose rows are contiguous 256-byte pieces.  Only whole halves are in the view.
-inline bool make_half_map(CUtensorMap* m, const float* base, int n, long long d, long long ld) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) return false;
-  const long long halves = d / kHalfCols;
-  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(kHalfCols), static_cast<cuuint64_t>(halves > 0 ? halves : 1),
-                              static_cast<cuuint64_t>(n)};
-  const cuuint64_t strides[2] = {kHalfCols * sizeof(float), static_cast<cuuint64_t>(ld) * sizeof(float)};
-  const cuuint32_t box[3] = {static_cast<cuuint32_t>(kHalfCols), 2, static_cast<cuuint32_t>(n)};
-  const cuuint32_t elem[3] = {1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, elem,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-__device__ __forceinline__ void slab_load(float* dst, const CUtensorMap* map, int half, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
-          s_addr(dst)),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(half), "r"(0), "r"(s_addr(bar))
-      : "memory");
-}
-
-__device__ __forceinline__ void slab_store(const CUtensorMap* map, int half, const float* src) {
-  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
-                   reinterpret_cast<uint64_t>(map)),
-               "r"(0), "r"(half), "r"(0), "r"(s_addr(src))
-               : "memory");
-}
-
-// 4 x 4 transpose over the four lanes that share a coordinate (lane bits 0 and 1): lane kq gives row kq = v[0..3]
-// and receives column kq.
-__device__ __forceinline__ void transpose_quad(float (&v)[4], int kq) {
-  const bool b0 = (kq & 1) != 0, b1 = (kq & 2) != 0;
-  float s0 = b0 ? v[0] : v[1], s1 = b0 ? v[2] : v[3];
-  float r0 = __shfl_xor_sync(0xffffffffu, s0, 1), r1 = __shfl_xor_sync(0xffffffffu, s1, 1);
-  if (b0) { v[0] = r0; v[2] = r1; } else { v[1] = r0; v[3] = r1; }
-  s0 = b1 ? v[0] : v[2];
-  s1 = b1 ? v[1] : v[3];
-  r0 = __shfl_xor_sync(0xffffffffu, s0, 2);
-  r1 = __shfl_xor_sync(0xffffffffu, s1, 2);
-  if (b1) { v[0] = r0; v[1] = r1; } else { v[2] = r0; v[3] = r1; }
-}
-
 // Transform of one worker column (this lane's R values along the block axis) into the Fourier components of the
 // block cycle, and back.  R = 8: butterflies of the real 8-point transform WITHOUT normalisation (20 operations
 // instead of 48; the host folds the two missing factors 1/8 resp. 1/4 into the per-frequency blocks).  Other R:
@@ -291,8 +246,8 @@ step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, co
         const bool any = half < halves;  // a slab without a whole half is served entirely by its lanes
         bar_expect_tx(&xy_full[sx], any ? Plan::kXYBytes : 0u);
         if (any) {
-          slab_load(tx, &maps.x, half, &xy_full[sx]);
-          slab_load(tx + Plan::kTileFloats, &maps.y, half, &xy_full[sx]);
+          rows_load(tx, &maps.x, half, 0, &xy_full[sx]);
+          rows_load(tx + Plan::kTileFloats, &maps.y, half, 0, &xy_full[sx]);
         }
       }
       if (!ok) {
@@ -320,9 +275,9 @@ step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, co
         const bool any = half < halves;
         bar_expect_tx(&e_full[se], any ? Plan::kEBytes : 0u);
         if (any) {
-          slab_load(te, &maps.g, half, &e_full[se]);
-          slab_load(te + Plan::kTileFloats, &maps.a, half, &e_full[se]);
-          slab_load(te + 2 * Plan::kTileFloats, &maps.c, half, &e_full[se]);
+          rows_load(te, &maps.g, half, 0, &e_full[se]);
+          rows_load(te + Plan::kTileFloats, &maps.a, half, 0, &e_full[se]);
+          rows_load(te + 2 * Plan::kTileFloats, &maps.c, half, 0, &e_full[se]);
         }
       }
       if (!ok) {
@@ -346,9 +301,9 @@ step_torus_kernel(const StepParams p, const __grid_constant__ TorusMaps maps, co
         const float* te = e_mem + static_cast<size_t>(se) * 3 * Plan::kTileFloats;  // now [g' | x' | y']
         const int half = static_cast<int>((blockIdx.x + k * gridDim.x) * 2);
         if (half < halves) {  // the stores clip at the last whole half
-          slab_store(&maps.gs, half, te);
-          slab_store(&maps.xs, half, te + Plan::kTileFloats);
-          slab_store(&maps.ys, half, te + 2 * Plan::kTileFloats);
+          rows_store(&maps.gs, half, 0, te);
+          rows_store(&maps.xs, half, 0, te + Plan::kTileFloats);
+          rows_store(&maps.ys, half, 0, te + 2 * Plan::kTileFloats);
         }
         store_commit();
         store_wait_read();  // the stage may be refilled now
@@ -519,9 +474,9 @@ bool torus_variant_available(int n) { return (n == 32 || n == 64) && encode_tile
 
 bool build_maps_torus(const StepParams& p, TensorMapSet* out) {
   TorusMaps& m = *reinterpret_cast<TorusMaps*>(out->bytes);
-  if (!make_half_map(&m.x, p.x, p.n, p.d, p.ld) || !make_half_map(&m.y, p.y, p.n, p.d, p.ld) ||
-      !make_half_map(&m.g, p.g, p.n, p.d, p.ld) || !make_half_map(&m.a, p.a, p.n, p.d, p.ld) ||
-      !make_half_map(&m.c, p.c, p.n, p.d, p.ld))
+  if (!make_half_map(&m.x, p.x, p.n, p.d, p.ld, p.n) || !make_half_map(&m.y, p.y, p.n, p.d, p.ld, p.n) ||
+      !make_half_map(&m.g, p.g, p.n, p.d, p.ld, p.n) || !make_half_map(&m.a, p.a, p.n, p.d, p.ld, p.n) ||
+      !make_half_map(&m.c, p.c, p.n, p.d, p.ld, p.n))
     return false;
   m.xs = m.x;
   m.ys = m.y;

@@ -60,6 +60,8 @@ def test_a_wait_that_nothing_ends_gives_up_and_is_reported():
     (48, 64 * 148 * 2 + 5, 2, B.DETAG_VARIANT_DENSE, 1),    # band kernel, dense window mode
     (64, 64 * 148 * 3 + 5, 2, B.DETAG_VARIANT_TORUS, 2),    # block-circulant transform kernel
     (32, 64 * 148 * 3 + 5, 2, B.DETAG_VARIANT_TORUS, 0),
+    (72, 64 * 148 * 2 + 5, 2, B.DETAG_VARIANT_DENSE, 1),    # dense kernel with the polynomial in registers, two stages of g, a, c
+    (128, 64 * 148 * 2 + 37, 2, B.DETAG_VARIANT_DENSE, 0),  # ... one stage
 ])
 def test_a_stalled_loader_times_out_every_waiter_and_the_state_recovers(n, d, K, variant, after):
     m, a, c, x0 = _case(n, d, n, torus=variant == B.DETAG_VARIANT_TORUS)

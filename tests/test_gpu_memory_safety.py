@@ -52,6 +52,7 @@ def _guarded_state(torch, m, d, ld, K, eta, observe, variant, where):
     (33, 67, 68, 2, B.DETAG_VARIANT_DENSE), (50, 130, 136, 3, B.DETAG_VARIANT_DENSE), (64, 65, 68, 2, B.DETAG_VARIANT_DENSE),
     (64, 67, 72, 4, B.DETAG_VARIANT_RING), (96, 130, 132, 2, B.DETAG_VARIANT_RING),
     (64, 67, 72, 4, B.DETAG_VARIANT_TORUS), (32, 130, 132, 2, B.DETAG_VARIANT_TORUS), (64, 3, 4, 2, B.DETAG_VARIANT_TORUS),
+    (72, 67, 68, 2, B.DETAG_VARIANT_DENSE), (100, 130, 132, 3, B.DETAG_VARIANT_DENSE), (128, 31, 32, 2, B.DETAG_VARIANT_DENSE),
     (9, 77, 80, 3, B.DETAG_VARIANT_CSR), (70, 33, 36, 2, B.DETAG_VARIANT_CSR)])
 def test_nothing_outside_the_arrays_is_written(n, d, ld, K, variant):
     import torch

@@ -305,6 +305,38 @@ def test_circulant_kernel_with_a_dense_polynomial(n, d, K, kind):
     _check_trajectory(m, K, eta, 0.02, a, c, x0, 0.1, 5, steps=4, variants=[B.DETAG_VARIANT_RING])
 
 
+@pytest.mark.parametrize("n,d,K,kind", [(100, 130, 6, "regular4"), (65, 67, 3, "ring"), (72, 1, 2, "regular4"),
+                                        (88, 31, 4, "regular4"), (96, 1057, 5, "directed"), (104, 64, 8, "regular4"),
+                                        (127, 97, 3, "path"), (128, 160, 12, "regular4")])
+def test_dense_polynomial_held_in_registers(n, d, K, kind):
+    """64 < n <= 128, any matrix: the polynomial as register-resident warp strips.  Unstructured, non-symmetric and
+    irregular matrices, worker counts on and off the 8-row blocks, d below, on and off the 32-column halves the
+    kernel takes (the remainder runs on the generic kernel in the same call)."""
+    rng = np.random.default_rng(n * 31 + d)
+    if kind == "regular4":
+        m = inputs.metropolis_weights(inputs.random_regular4_graph(n, n + K))
+    elif kind == "ring":
+        m = inputs.metropolis_weights(inputs.ring_graph(n))
+    elif kind == "path":
+        m = inputs.metropolis_weights(inputs.path_graph(n))
+    else:
+        m = inputs.directed_cycle_blend(n, 0.4, 0.35)
+    eta = orc.spectrum(m.to_dense()).eta if kind != "directed" else 0.3
+    st = B.detag_create(n, d, m.row_ptr, m.col_idx, m.vals, K, eta, 0.05)
+    try:
+        picked = B.detag_get_variant(st)
+    finally:
+        B.detag_destroy(st)
+    if kind in ("regular4", "path"):
+        assert picked == B.DETAG_VARIANT_DENSE  # no structure: the dense polynomial is the default
+    a, c = _random_objective(rng, n, d, scale=0.1)
+    x0 = rng.standard_normal((n, d)).astype(np.float32)
+    variants = [B.DETAG_VARIANT_DENSE]
+    _check_one_step(m, K, eta, 0.02, a, c, x0, 0.1, 23, variants=variants)
+    _check_one_step(m, K, eta, 0.02, a, c, x0, 0.1, 23, j0=(3 << 32) - 40, variants=variants)
+    _check_trajectory(m, K, eta, 0.02, a, c, x0, 0.1, 23, steps=5, variants=variants)
+
+
 def test_misuse_is_reported_not_faulted():
     import torch
 

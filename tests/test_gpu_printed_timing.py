@@ -105,6 +105,17 @@ def test_ring_band_kernel(n, d, K):
     _check_trajectory(m, K, 0.3, 0.02, a, c, x0, 0.1, 5, 5, [B.DETAG_VARIANT_RING])
 
 
+@pytest.mark.parametrize("n,d,K", [(100, 131, 4), (72, 64, 3)])
+def test_register_resident_dense_kernel(n, d, K):
+    rng = np.random.default_rng(n + d)
+    m = inputs.metropolis_weights(inputs.random_regular4_graph(n, 3))
+    eta = orc.spectrum(m.to_dense()).eta
+    a, c = _objective(rng, n, d, scale=0.1)
+    x0 = rng.standard_normal((n, d)).astype(np.float32)
+    _check_one_phase(m, K, eta, 0.02, a, c, x0, 0.1, 5, [B.DETAG_VARIANT_DENSE, B.DETAG_VARIANT_CSR])
+    _check_trajectory(m, K, eta, 0.02, a, c, x0, 0.1, 5, 5, [B.DETAG_VARIANT_DENSE])
+
+
 def test_first_phase_differs_from_the_default_step_only_in_the_gradient():
     """From the common initial state both gradient points give the same x' (bit for bit); the gradients differ."""
     rng = np.random.default_rng(3)
