@@ -38,6 +38,7 @@ BYTES_PER_WC = 32  # read x, y, g, a, c + write x, y, g, float32 each: the fused
 # small case of the same kernel; traffic grows in proportion to n*d).  Keyed by the sha256 prefix of the kernel
 # sources the capture was taken on: a changed kernel reports null until it is captured again.
 KERNEL_SOURCES = {
+    "wide": ("step_wide.cu", "pipeline.cuh", "noise.cuh"),
     "mma": ("step_mma.cu", "mma_common.cuh", "pipeline.cuh", "noise.cuh"),
     "band": ("step_band.cu", "pipeline.cuh", "noise.cuh"),
     "ring": ("step_ring.cu", "pipeline.cuh", "noise.cuh"),
@@ -334,40 +335,51 @@ def theorem3_regime(dev, args) -> dict:
 
 
 def general_graph(dev, args) -> dict:
-    """A graph none of the structured kernels takes - 100 workers on a seeded random 4-regular graph, K = 6,
-    d = 2,000,000 - through the generic rounds kernel: its step time and roofline fraction."""
+    """Graphs none of the structured kernels takes - seeded random 4-regular graphs with 100 and with 72 workers,
+    K = 6, d = 2,000,000: step time and roofline fractions of the kernel the library picks (the dense polynomial
+    held in registers, whose bound is the FP64 tensor pipe: 2 * n_padded multiply-adds per worker-coordinate) and,
+    for the 100-worker graph, of the generic rounds kernel that takes every graph."""
     import torch
 
     from paper_2006_08085_b200 import binding as B
     from paper_2006_08085_b200.session import Session
 
-    n, d, K = 100, 2_000_000, 6
-    gm = inputs.metropolis_weights(inputs.random_regular4_graph(n, 7))
-    s = Session(gm, d, K, float("nan"), 0.001, None, None, None, 0.1, 7, device=str(dev))
-    gen = torch.Generator(device=dev).manual_seed(7)
-    s.a.uniform_(0.5, 2.0, generator=gen)  # objective data drawn on the device: this leg times the kernel only
-    s.c.normal_(generator=gen)
-    stream = torch.cuda.current_stream(dev)
-    s.init()
-    for _ in range(3):
-        B.detag_step(s.state, stream)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(10):
-        B.detag_step(s.state, stream)
-    e1.record(stream)
-    torch.cuda.synchronize(dev)
-    s.status()
-    ms = e0.elapsed_time(e1) / 10
-    variant = VARIANT_NAMES.get(B.detag_get_variant(s.state), "other")
-    s.close()
-    del s
-    torch.cuda.empty_cache()
+    d, K = (args.d if args.leg == "general_graph" and args.d else 2_000_000), 6
     peak, _ = measured_peak_gbs()
-    gbs = BYTES_PER_WC * n * d / (ms * 1e-3) / 1e9
-    return {"workload": "100 workers, random 4-regular graph (Metropolis weights), d = 2,000,000, K = 6", "variant": variant,
-            "ms_per_step": ms, "value": n * d / (ms * 1e-3), "unit": UNIT, "achieved_gbs": gbs,
-            "frac_of_measured_peak": gbs / peak, "frac_of_8TBps_nominal": gbs / 8000.0}
+    stream = torch.cuda.current_stream(dev)
+
+    def one(n: int, forced: int) -> dict:
+        gm = inputs.metropolis_weights(inputs.random_regular4_graph(n, 7))
+        s = Session(gm, d, K, float("nan"), 0.001, None, None, None, 0.1, 7, device=str(dev), variant=forced)
+        gen = torch.Generator(device=dev).manual_seed(7)
+        s.a.uniform_(0.5, 2.0, generator=gen)  # objective data drawn on the device: this leg times the kernel only
+        s.c.normal_(generator=gen)
+        s.init()
+        for _ in range(3):
+            B.detag_step(s.state, stream)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(10):
+            B.detag_step(s.state, stream)
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        s.status()
+        ms = e0.elapsed_time(e1) / 10
+        variant = VARIANT_NAMES.get(B.detag_get_variant(s.state), "other")
+        s.close()
+        del s
+        torch.cuda.empty_cache()
+        gbs = BYTES_PER_WC * n * d / (ms * 1e-3) / 1e9
+        out = {"workload": f"{n} workers, random 4-regular graph (Metropolis weights), d = {d:,}, K = {K}",
+               "variant": variant, "ms_per_step": ms, "value": n * d / (ms * 1e-3), "unit": UNIT, "achieved_gbs": gbs,
+               "frac_of_measured_peak": gbs / peak, "frac_of_8TBps_nominal": gbs / 8000.0}
+        if variant == "dense":
+            fma = 2 * ((n + 7) // 8 * 8)
+            out["fp64_fma_per_wc"] = fma
+            out["fp64_pipe_frac"] = fma * out["value"] / (FP64_FMA_PER_CLK_SM * SM_COUNT * 1965e6)
+        return out
+
+    return {"picked_100": one(100, 0), "rounds_100": one(100, B.DETAG_VARIANT_CSR), "picked_72": one(72, 0)}
 
 
 def run_host_only(args, rank: int, world: int) -> None:
@@ -415,6 +427,10 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    if args.leg == "general_graph":  # that leg alone (a small case of it with --d: what the ncu capture runs)
+        if rank == 0:
+            print(json.dumps({"general_graph": general_graph(dev, args)}), flush=True)
+        return
     cfg = inputs.CONFIGS[args.config]
     if args.d:
         cfg = cfg.with_d(args.d)
@@ -630,6 +646,7 @@ def main() -> None:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--no-modes", action="store_true", help="skip the D-PSGD and caller-written-gradient legs")
+    ap.add_argument("--leg", default="", choices=["", "general_graph"], help="run this extra leg alone")
     ap.add_argument("--host-only", action="store_true",
                     help="multi-rank plumbing only (gloo, no CUDA call): what the CPU test of --gpus N runs")
     args = ap.parse_args()

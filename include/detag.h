@@ -58,7 +58,8 @@ enum {
 enum {
   DETAG_VARIANT_AUTO = 0,  /* host cost model picks */
   DETAG_VARIANT_CSR = 1,   /* K rounds of neighbour-indexed sums over the CSR rows, slab staged on chip: any graph, n <= 1024 */
-  DETAG_VARIANT_DENSE = 2, /* one product with the host-precomputed polynomial P_K(M), n <= 64 */
+  DETAG_VARIANT_DENSE = 2, /* one product with the host-precomputed polynomial P_K(M), n <= 128 (any M); for 64 < n <= 128
+                              the last d % 32 coordinates run through the CSR kernel in the same call */
   DETAG_VARIANT_RING = 3,  /* circulant M (rings), n % 32 == 0, 64 <= n <= 1024: the circulant polynomial P_K(M) as a band
                               while K * bandwidth <= 16, as a dense circulant (n <= 256) beyond, e.g. at Theorem 3's phase
                               length; the last d % 64 coordinates run through the CSR kernel in the same call */

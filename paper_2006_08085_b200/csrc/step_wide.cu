@@ -20,9 +20,11 @@
 // A warp works through the slab two 8-coordinate tiles at a time: four independent accumulator chains (model and
 // tracker of both tiles) of ceil(n / 4) MMAs each, then the tail of those 2 x 2 x 8 elements.  The four lanes of a
 // coordinate share the Philox calls of the tail: the two tiles' two 4-worker quads make four calls, one per lane,
-// handed round by a 4 x 4 transpose.
+// handed round by a 4 x 4 transpose.  The FP64 MMA rate of each of the SM's four warp schedulers is what bounds the
+// kernel (2 n multiply-adds per element against 32 bytes), so the blocks are dealt to the schedulers evenly: see
+// wide_consumers().
 //
-// Roles of the persistent CTA (one per SM): ceil(n / 8) consumer warps; a loader for x, y (two stages, handed back when
+// Roles of the persistent CTA (one per SM): ceil(n / 8) or a few more consumer warps; a loader for x, y (two stages, handed back when
 // every warp has finished the slab's contractions); a loader for g, a, c (two stages while ten tiles fit in shared
 // memory, n <= 88, else one); a storer that sends a finished stage out with three TMA stores.  Every wait is bounded.
 //
@@ -51,9 +53,15 @@ struct WideMaps {
 };
 static_assert(sizeof(WideMaps) <= sizeof(TensorMapSet), "tensor map storage");
 
+// Consumer warps for B output blocks.  A warp scheduler's share of the MMAs is what bounds the kernel, and warps go to
+// the four schedulers round robin: with B = 4m + 1 blocks the last block is shared by four warps (one pair of tiles
+// each), with B = 4m + 2 the last two blocks by two warps each (two pairs each), so that every scheduler carries the
+// same load; B = 4m + 3 is left as it is (one scheduler a quarter block short).
+__host__ __device__ constexpr int wide_consumers(int blocks) { return blocks % 4 == 1 ? blocks + 3 : blocks % 4 == 2 ? blocks + 2 : blocks; }
+
 struct WidePlan {
   int rows;       // n rounded up to a multiple of 8
-  int warps;      // consumer warps = rows / 8
+  int warps;      // consumer warps
   int e_stages;   // 1 or 2
   int tile_floats;
   size_t ctrl_offset, smem_bytes;
@@ -62,7 +70,7 @@ struct WidePlan {
 inline WidePlan wide_plan(int n) {
   WidePlan w{};
   w.rows = (n + 7) / 8 * 8;
-  w.warps = w.rows / 8;
+  w.warps = wide_consumers(w.rows / 8);
   w.tile_floats = w.rows * kWS;
   const size_t tile = static_cast<size_t>(w.tile_floats) * 4;
   w.e_stages = (2 * kWXYStages + 6) * tile + 128 + 1024 <= kWSmemLimit ? 2 : 1;
@@ -73,14 +81,19 @@ inline WidePlan wide_plan(int n) {
 
 // kKs: k-steps issued, ceil(n / 4) rounded up to an even number (the B fragments beyond n are zero).
 template <int kKs>
-__global__ void __launch_bounds__((kKs / 2 + 3) * 32, 1)
+__global__ void __launch_bounds__((wide_consumers(kKs / 2) + 3) * 32, 1)
 step_wide_kernel(const StepParams p, const __grid_constant__ WideMaps maps, const double* __restrict__ p_frag,
                  const int rows, const int e_stages) {
   extern __shared__ unsigned char smem_unaligned[];
   // the swizzle pattern is a function of the shared-memory address: tiles start on 1 KiB boundaries
   unsigned char* smem_raw = smem_unaligned + ((1024u - (s_addr(smem_unaligned) & 1023u)) & 1023u);
   const int tile_floats = rows * kWS;
-  const int consumers = rows / 8;
+  constexpr int kBlocks = kKs / 2;                      // 8-worker output blocks
+  constexpr int consumers = wide_consumers(kBlocks);
+  // Tail of a pair of tiles in one instruction stream with the next pair's contractions: pays only at the smallest
+  // size (measured, d = 2 M: 1.68 against 1.79 ms at n = 72; 2.09 against 2.06 at n = 80, 2.99 against 2.96 at n = 96),
+  // and needs the 128 registers per thread that 16 warps leave.
+  constexpr bool kPipelined = kKs <= 18;
   float* xy_mem = reinterpret_cast<float*>(smem_raw);            // [stage][x | y]
   float* e_mem = xy_mem + kWXYStages * 2 * tile_floats;          // [stage][g | a | c]
   uint64_t* xy_full = reinterpret_cast<uint64_t*>(e_mem + e_stages * 3 * tile_floats);
@@ -187,16 +200,26 @@ step_wide_kernel(const StepParams p, const __grid_constant__ WideMaps maps, cons
     return;
   }
 
-  // ------------------------------------------------------------------ consumer warp: output workers 8 warp .. 8 warp + 7
+  // ------------------------------------------------------------------ consumer warp: output workers 8 block .. 8 block + 7
+  // for num_pairs of the slab's four pairs of tiles, from first_pair on
+  int block = warp, first_pair = 0, num_pairs = kWPairs;
+  if (kBlocks % 4 == 1 && warp >= kBlocks - 1) {
+    block = kBlocks - 1;
+    first_pair = warp - (kBlocks - 1);
+    num_pairs = 1;
+  } else if (kBlocks % 4 == 2 && warp >= kBlocks - 2) {
+    block = kBlocks - 2 + ((warp - (kBlocks - 2)) >> 1);
+    first_pair = 2 * ((warp - (kBlocks - 2)) & 1);
+    num_pairs = 2;
+  }
   const int kq = lane & 3, crow = lane >> 2;  // crow: this lane's coordinate within an 8-coordinate tile
   double bf[kKs];                             // this warp's strip of P in fragment order
 #pragma unroll
-  for (int s = 0; s < kKs; ++s) bf[s] = p_frag[(static_cast<size_t>(warp) * 32 + s) * 32 + lane];
+  for (int s = 0; s < kKs; ++s) bf[s] = p_frag[(static_cast<size_t>(block) * 32 + s) * 32 + lane];
   const double alpha = p.alpha;
   const float sigma = static_cast<float>(p.sigma);
-  const bool noisy = p.sigma != 0.0;
   const bool at_start = p.grad_at_start != 0;
-  const uint32_t quad = 2u * static_cast<uint32_t>(warp) + (kq & 1);  // the Philox quad this lane draws for its coordinate group
+  const uint32_t quad = 2u * static_cast<uint32_t>(block) + (kq & 1);  // the Philox quad this lane draws for its coordinate group
   // Float offset, inside an array's tile, of this lane's element of row kq in 8-coordinate tile o: tile = [row][half][32],
   // the 16-byte chunk index XORed with the low three bits of the 128-byte row number 2 row + half (the tensor maps'
   // swizzle), which is 2 kq + half for every row kq + 4 m.  Row kq + 4 m lies m * 256 floats further.
@@ -220,49 +243,40 @@ step_wide_kernel(const StepParams p, const __grid_constant__ WideMaps maps, cons
     float* sa = sg + tile_floats;
     float* sc = sa + tile_floats;
     const long long j0 = (blockIdx.x + static_cast<long long>(k) * gridDim.x) * kWS;
-    bool e_seen = false;
-
-#pragma unroll 1
-    for (int pair = 0; pair < kWPairs; ++pair) {
-      if (j0 + pair * 16 >= p.d) break;  // tiles wholly beyond column d compute nothing
+    // The four accumulator chains of a pair of tiles: model and tracker of both.
+    auto contract = [&](int pair, double (&cx)[2][2], double (&cy)[2][2]) {
       const int off0 = tile_off(2 * pair), off1 = tile_off(2 * pair + 1);
-      double cx0[2] = {0.0, 0.0}, cy0[2] = {0.0, 0.0}, cx1[2] = {0.0, 0.0}, cy1[2] = {0.0, 0.0};
+      cx[0][0] = cx[0][1] = cx[1][0] = cx[1][1] = 0.0;
+      cy[0][0] = cy[0][1] = cy[1][0] = cy[1][1] = 0.0;
 #pragma unroll
       for (int s = 0; s < kKs; ++s) {
         const double ax0 = static_cast<double>(sxp[off0 + s * 256]), ay0 = static_cast<double>(syp[off0 + s * 256]);
         const double ax1 = static_cast<double>(sxp[off1 + s * 256]), ay1 = static_cast<double>(syp[off1 + s * 256]);
-        dmma(cx0, ax0, bf[s]);
-        dmma(cy0, ay0, bf[s]);
-        dmma(cx1, ax1, bf[s]);
-        dmma(cy1, ay1, bf[s]);
+        dmma(cx[0], ax0, bf[s]);
+        dmma(cy[0], ay0, bf[s]);
+        dmma(cx[1], ax1, bf[s]);
+        dmma(cy[1], ay1, bf[s]);
       }
-      if (!e_seen) {  // g, a, c are needed from here on; their loads had the first contractions to arrive in
-        if (lane == 0) ok = bar_wait(&e_full[se], (k / e_stages) & 1, limit);
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) {
-          if (lane == 0) atomicExch(p.status, 1);
-          return;
-        }
-        e_seen = true;
-      }
-      // ---- tail of the 2 tiles x 2 workers of this lane
-      float xi[4] = {0.f, 0.f, 0.f, 0.f};
-      if (noisy) {
-        // lane kq draws quad 2 warp + (kq & 1) at the coordinate of tile (kq >> 1); the transpose hands lane kq
-        // position kq of all four: xi[i] belongs to worker 8 warp + 4 (i & 1) + kq in tile (i >> 1)
-        const unsigned long long jn = static_cast<unsigned long long>(p.coord_offset + j0 + pair * 16 + (kq >> 1) * 8 + crow);
-        normal_quad(p.seed_lo, p.seed_hi, jn, quad, p.t_noise, xi);
-        transpose_quad(xi, kq);
-      }
+    };
+    // Normals of the pair's 2 tiles x 2 workers of this lane: lane kq draws quad 2 block + (kq & 1) at the coordinate of
+    // tile (kq >> 1); the transpose hands lane kq position kq of all four, so that xi[i] belongs to worker
+    // 8 block + 4 (i & 1) + kq in tile (i >> 1).
+    auto draw = [&](int pair, float (&xi)[4]) {
+      const unsigned long long jn = static_cast<unsigned long long>(p.coord_offset + j0 + pair * 16 + (kq >> 1) * 8 + crow);
+      normal_quad(p.seed_lo, p.seed_hi, jn, quad, p.t_noise, xi);
+      transpose_quad(xi, kq);
+    };
+    // Element-wise tail of the pair: model update, gradient, tracker fold; g', x', y' go over g, a, c.
+    auto tail = [&](int pair, const double (&cx)[2][2], const double (&cy)[2][2], const float (&xi)[4]) {
 #pragma unroll
       for (int t = 0; t < 2; ++t) {
-        const int off = (t == 0 ? off0 : off1) + warp * 512;
+        const int off = tile_off(2 * pair + t) + block * 512;
         const long long j = j0 + pair * 16 + t * 8 + crow;
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const int o = off + e * 256;
-          const double xt = t == 0 ? cx0[e] : cx1[e], yt = t == 0 ? cy0[e] : cy1[e];
-          const float xo = static_cast<float>(fma(-alpha, yt, xt));  // x' = x~ - alpha y~, rounded once
+          const double yt = cy[t][e];
+          const float xo = static_cast<float>(fma(-alpha, yt, cx[t][e]));  // x' = x~ - alpha y~, rounded once
           const float x_at = at_start ? sxp[o] : xo;  // Algorithm 2 as printed: the gradient at the model the step started from
           const float gold = sg[o];
           const float go = fmaf(sa[o], x_at - sc[o], sigma * xi[2 * t + e]);
@@ -270,22 +284,70 @@ step_wide_kernel(const StepParams p, const __grid_constant__ WideMaps maps, cons
           sg[o] = go;
           sa[o] = xo;
           sc[o] = yo;
-          const int row = 8 * warp + kq + 4 * e;
+          const int row = 8 * block + kq + 4 * e;
           if (p.y_obs != nullptr && row < p.n && j < p.d)  // optional observer: the gossiped tracker, stored directly
             p.y_obs[static_cast<long long>(row) * p.ld + j] = static_cast<float>(yt);
         }
       }
-    }
-    __syncwarp();
-    if (lane == 0) bar_arrive(&xy_empty[sx]);  // the x, y stage can be refilled
-    if (!e_seen) {  // a slab wholly beyond column d (cannot happen with the launcher's slab count): keep the protocol
-      if (lane == 0) ok = bar_wait(&e_full[se], (k / e_stages) & 1, limit);
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      if (!ok) {
+    };
+    auto wait_e = [&]() {  // g, a, c are needed from the first tail on; their loads had the first contractions to arrive in
+      bool got = true;
+      if (lane == 0) got = bar_wait(&e_full[se], (k / e_stages) & 1, limit);
+      return __shfl_sync(0xffffffffu, got ? 1 : 0, 0) != 0;
+    };
+
+    // pairs of tiles of this slab that are this warp's: the slab has all four or (the last one, d a multiple of 32) two
+    const int slab_pairs = p.d - j0 >= kWS ? kWPairs : kWPairs / 2;
+    const int my_pairs = slab_pairs - first_pair < num_pairs ? slab_pairs - first_pair : num_pairs;
+    double cx[2][2], cy[2][2];
+    if (kPipelined && my_pairs == kWPairs) {
+      // Software pipeline: the tail of a pair (a long dependent chain: Philox, Box-Muller, special-function unit)
+      // shares straight-line code with the contractions of the next pair, whose MMAs fill its issue slots.
+      contract(0, cx, cy);
+      if (!wait_e()) {
+        if (lane == 0) atomicExch(p.status, 1);
+        return;
+      }
+#pragma unroll
+      for (int pair = 1; pair <= kWPairs; ++pair) {
+        float xi[4];
+        draw(pair - 1, xi);
+        double nx[2][2], ny[2][2];
+        if (pair < kWPairs) contract(pair, nx, ny);
+        tail(pair - 1, cx, cy, xi);
+        if (pair < kWPairs) {
+#pragma unroll
+          for (int t = 0; t < 2; ++t)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              cx[t][e] = nx[t][e];
+              cy[t][e] = ny[t][e];
+            }
+        }
+      }
+    } else {
+      bool e_seen = false;
+#pragma unroll 1
+      for (int q = 0; q < my_pairs; ++q) {
+        contract(first_pair + q, cx, cy);
+        if (!e_seen) {
+          e_seen = true;
+          if (!wait_e()) {
+            if (lane == 0) atomicExch(p.status, 1);
+            return;
+          }
+        }
+        float xi[4];
+        draw(first_pair + q, xi);
+        tail(first_pair + q, cx, cy, xi);
+      }
+      if (!e_seen && !wait_e()) {  // nothing of this slab is this warp's: keep the protocol
         if (lane == 0) atomicExch(p.status, 1);
         return;
       }
     }
+    __syncwarp();
+    if (lane == 0) bar_arrive(&xy_empty[sx]);  // the x, y stage can be refilled
     fence_async_shared();  // results visible to the TMA stores
     __syncwarp();
     if (lane == 0) bar_arrive(&out_ready[se]);
