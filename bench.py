@@ -47,6 +47,10 @@ KERNEL_SOURCES = {
 }
 MEASURED_TRAFFIC = {
     # (kernel, mode): (source digest, bytes per wc)
+    ("mma", "dense"): ("22eae46feb506e80", 31.46),     # cfg5 shape at d = 2 M: 1.2949 GB read + 0.7183 GB written / 64 M wc
+    ("torus", "torus8"): ("427a2bff49b63d9c", 31.27),  # cfg3 shape at d = 1 M: 1.2803 + 0.7208 GB / 64 M wc
+    ("ring", "band"): ("60c16ee651aa8e4f", 31.12),     # cfg4 shape at d = 200 k: 1.0280 + 0.5652 GB / 51.2 M wc
+    ("wide", "dense"): ("77d5b7be943b4c42", 30.83),    # 100-worker random graph at d = 400 k: 0.8011 + 0.4321 GB / 40 M wc
 }
 
 # Float64 multiply-adds per worker-coordinate on the FP64 pipe (both contractions, padded shapes) and that
@@ -60,7 +64,7 @@ SM_COUNT = 148
 
 def kernel_key(variant: str, n: int):
     if variant == "dense":
-        return ("mma", "dense") if n <= 32 else ("band", "dense")
+        return ("mma", "dense") if n <= 32 else ("band", "dense") if n <= 64 else ("wide", "dense")
     if variant == "ring":
         return ("ring", "band")
     if variant == "csr":
