@@ -478,7 +478,8 @@ def test_cfg3_full_size_sampled_blocks():
 
 
 # ----------------------------------------------------------------------------- host-resident stepping
-@pytest.mark.parametrize("n,d,K,graph", [(16, 100_003, 4, "ring"), (64, 20_000, 3, "ring"), (9, 5_001, 2, "path")])
+@pytest.mark.parametrize("n,d,K,graph", [(16, 100_003, 4, "ring"), (64, 20_000, 3, "ring"), (9, 5_001, 2, "path"),
+                                         (100, 17_003, 2, "path")])
 def test_step_host_matches_device_resident_stepping(n, d, K, graph):
     """detag_step_host (state in page-locked host memory, chunked through a device staging area) performs the
     same arithmetic per coordinate as detag_step: bit-identical results, several chunks and a ragged last one."""
