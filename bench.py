@@ -291,6 +291,8 @@ def time_config(name: str, dev, args) -> dict:
     if key in FP64_FMA_PER_WC:
         out["fp64_fma_per_wc"] = FP64_FMA_PER_WC[key]
         out["fp64_pipe_frac"] = FP64_FMA_PER_WC[key] * out["value"] / (FP64_FMA_PER_CLK_SM * SM_COUNT * 1965e6)
+    traffic = measured_traffic_bytes(variant, cfg.n, cfg.wc)  # ncu DRAM bytes of a small case, scaled; None if stale
+    out["traffic_bytes_per_step"] = traffic
     return out
 
 
