@@ -26,6 +26,7 @@ struct StepParams {
   int K;
   int S;           // slab width in coordinates (power of two)
   int log2S;
+  int csr_sub;     // generic rounds kernel: independent pieces the slab is cut into
   long long d;
   long long ld;
   long long num_slabs;

@@ -9,12 +9,19 @@
 //      all eight values), the thread's own previous values never leave its registers; a barrier separates reading
 //      a round's inputs from overwriting them, so one slab buffer per array suffices;
 //   3. it finishes the step element-wise (Algorithm 2): x' = x~ - alpha y~, the stochastic gradient
-//      g' = a (x' - c) + sigma xi at the new model (the four workers of a Philox call sit in four neighbouring lanes:
+//      g' = a (x' - c) + sigma xi at the new model (the four workers of a Philox call sit in four lanes of one warp:
 //      each lane draws one of the four coordinates and a 4 x 4 transpose hands everybody its own row), and the
 //      tracker fold y' = y~ + g' - g with the float32 value of g' that is stored, so that the stored tracker
 //      telescopes exactly against the stored gradients; a, c, g are 16-byte loads, x', y', g' 16-byte stores.
 // All on-chip arithmetic is float64; each result is rounded once when it is stored.  What bounds the kernel is the
-// shared-memory traffic of step 2: 8 bytes per multiply-add.
+// shared-memory traffic of step 2: 8 bytes per multiply-add.  Layout for that traffic: the threads of a worker
+// are neighbouring lanes (coordinate group fastest), and a slab row keeps the first coordinate pair of all groups
+// contiguously, then the second pairs: a 16-byte read per lane then covers 128 contiguous bytes of ONE row per
+// quarter warp - every bank once, whatever row the neighbour index names (with the thread's four doubles side by
+// side each of the two reads would use half of the banks, and four rows would meet in every quarter warp).  With
+// fewer than eight groups (n > 128) a quarter warp reads 2, 4 or 8 rows; the two pairs of a row then swap places
+// according to one bit of the row index, chosen so that consecutive rows - the neighbours of consecutive workers
+// on rings, tori and other banded matrices - fall on different banks.
 //
 // Modes: with caller-written gradients step 1 also applies Algorithm 2's tracker update, y + g_new - g_old, and
 // step 3 stores the gossiped tracker and copies g_new over g_old instead of evaluating a gradient; in D-PSGD
@@ -29,24 +36,25 @@ namespace detag {
 namespace {
 
 constexpr int kCsrThreads = 1024;
-constexpr int kCsrPad = 4;  // doubles of padding per slab row: neighbouring rows start 8 banks apart
+constexpr int kCsrPad = 0;  // contiguous 128-byte pieces need no padding
+constexpr int kCsrMaxS = 32;  // at most 8 coordinate groups: the four workers of a Philox call stay in one warp
 
 __host__ __device__ inline size_t csr_smem_bytes(int n, int nnz, int S, bool tables) {
-  // the x and y slabs + (if they fit) values, row pointers and columns
+  // the x and y slabs (S coordinates in all, in pieces or not) + (if they fit) values, row pointers and columns
   return static_cast<size_t>(2) * n * (S + kCsrPad) * sizeof(double) +
          (tables ? static_cast<size_t>(nnz) * sizeof(double) + static_cast<size_t>(n + 1 + nnz) * sizeof(int32_t) : 0);
 }
 
-// 4 x 4 transpose over the four lanes that share a coordinate group (lane bits 0 and 1).
-__device__ __forceinline__ void transpose_rows(float (&v)[4], int r4) {
+// 4 x 4 transpose over the four lanes that share a coordinate group: rows r4 = 0..3 sit `stride` lanes apart.
+__device__ __forceinline__ void transpose_rows(float (&v)[4], int r4, int stride) {
   const bool b0 = (r4 & 1) != 0, b1 = (r4 & 2) != 0;
   float s0 = b0 ? v[0] : v[1], s1 = b0 ? v[2] : v[3];
-  float r0 = __shfl_xor_sync(0xffffffffu, s0, 1), r1 = __shfl_xor_sync(0xffffffffu, s1, 1);
+  float r0 = __shfl_xor_sync(0xffffffffu, s0, stride), r1 = __shfl_xor_sync(0xffffffffu, s1, stride);
   if (b0) { v[0] = r0; v[2] = r1; } else { v[1] = r0; v[3] = r1; }
   s0 = b1 ? v[0] : v[2];
   s1 = b1 ? v[1] : v[3];
-  r0 = __shfl_xor_sync(0xffffffffu, s0, 2);
-  r1 = __shfl_xor_sync(0xffffffffu, s1, 2);
+  r0 = __shfl_xor_sync(0xffffffffu, s0, 2 * stride);
+  r1 = __shfl_xor_sync(0xffffffffu, s1, 2 * stride);
   if (b1) { v[0] = r0; v[1] = r1; } else { v[2] = r0; v[3] = r1; }
 }
 
@@ -71,17 +79,20 @@ __device__ __forceinline__ void store4(float* base, long long off, long long j, 
 }
 
 // kTables: the CSR arrays are read from shared memory (they fit) instead of global memory.
-template <bool kTables>
+// kSwap: fewer than eight coordinate groups, the pairs of a row swap places by a bit of the row index.
+template <bool kTables, bool kSwap>
 __global__ void __launch_bounds__(kCsrThreads, 1) step_csr_kernel(const StepParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int n = p.n, S = p.S, pitch = S + kCsrPad, tid = threadIdx.x;
+  // S coordinates per slab in p.csr_sub independent pieces of W = S / p.csr_sub coordinates (each with its own rows
+  // in shared memory): small graphs fill the thread block with several pieces
+  const int n = p.n, S = p.S, W = S / p.csr_sub, pitch = W + kCsrPad, tid = threadIdx.x;
   double* sx = reinterpret_cast<double*>(smem_raw);
-  double* sy = sx + static_cast<size_t>(n) * pitch;
+  double* sy = sx + static_cast<size_t>(p.csr_sub) * n * pitch;
   const double* vals = p.vals;
   const int32_t* rows = p.row_ptr;
   const int32_t* cols = p.col_idx;
   if (kTables) {
-    double* s_val = sy + static_cast<size_t>(n) * pitch;
+    double* s_val = sy + static_cast<size_t>(p.csr_sub) * n * pitch;
     int32_t* s_row = reinterpret_cast<int32_t*>(s_val + p.nnz);
     int32_t* s_col = s_row + (n + 1);
     for (int k = tid; k < p.nnz; k += kCsrThreads) {
@@ -94,21 +105,27 @@ __global__ void __launch_bounds__(kCsrThreads, 1) step_csr_kernel(const StepPara
     cols = s_col;
     __syncthreads();  // the tables are read right below
   }
-  // item = ((row quad * groups + coordinate group) * 4 + row within quad): the four rows of a Philox call in
-  // four neighbouring lanes
-  const int groups = S >> 2;
-  const int r4 = tid & 3, cg = (tid >> 2) % groups, q = (tid >> 2) / groups;
+  // item = ((row quad * 4 + row within quad) * groups + coordinate group): a row's threads side by side, the four
+  // rows of a Philox call `groups` lanes apart in one warp (groups is a power of two, at most 8)
+  const int groups = W >> 2, half = W >> 1, quads = (n + 3) / 4;
+  const int cg = tid & (groups - 1), r4 = (tid / groups) & 3, qs = (tid / groups) >> 2;
+  const int sub = qs / quads, q = qs - sub * quads;  // piece of the slab, row quad
   const int i = 4 * q + r4;
-  const bool owner = q < (n + 3) / 4 && i < n;  // threads without an element idle (they still meet the barriers)
+  const bool owner = sub < p.csr_sub && i < n;  // threads without an element idle (they still meet the barriers)
   const int k0 = owner ? rows[i] : 0, k1 = owner ? rows[i + 1] : 0;
   const double one_plus_eta = 1.0 + p.eta, eta = p.eta, alpha = p.alpha;
   const float sigma = static_cast<float>(p.sigma);
   const bool dpsgd = p.mode == kModeDpsgd, external = p.mode == kModeExternal;
-  double* my_x = sx + static_cast<size_t>(owner ? i : 0) * pitch + 4 * cg;
-  double* my_y = sy + static_cast<size_t>(owner ? i : 0) * pitch + 4 * cg;
+  // the thread's coordinates 4 cg .. 4 cg + 3: the first pair at 2 cg of the row, the second at half + 2 cg
+  const size_t piece = static_cast<size_t>(owner ? sub : 0) * n * pitch;
+  // which of a row's pairs comes first: bit log2(4 / groups) of the row index (8 groups: always the first pair)
+  const int swz_shift = groups >= 4 ? 0 : (groups == 2 ? 1 : 2), swz_mask = kSwap ? 1 : 0;
+  const int my_first = (((owner ? i : 0) >> swz_shift) & swz_mask) * half;   // offset of this thread's first pair
+  double* my_x = sx + piece + static_cast<size_t>(owner ? i : 0) * pitch + 2 * cg;
+  double* my_y = sy + piece + static_cast<size_t>(owner ? i : 0) * pitch + 2 * cg;
 
   for (long long slab = blockIdx.x; slab < p.num_slabs; slab += gridDim.x) {
-    const long long j = slab * S + 4 * cg;  // this thread's first coordinate
+    const long long j = slab * S + sub * W + 4 * cg;  // this thread's first coordinate
     const long long off = static_cast<long long>(i) * p.ld + j;
     const bool active = owner && j < p.d;
     double px[4], py[4];  // z_{r-1} of this thread's elements; z_r is in the slab
@@ -140,10 +157,10 @@ __global__ void __launch_bounds__(kCsrThreads, 1) step_csr_kernel(const StepPara
     }
     __syncthreads();  // the previous slab's rounds have finished reading the slab
     if (owner) {
-      *reinterpret_cast<double2*>(my_x) = make_double2(px[0], px[1]);
-      *reinterpret_cast<double2*>(my_x + 2) = make_double2(px[2], px[3]);
-      *reinterpret_cast<double2*>(my_y) = make_double2(py[0], py[1]);
-      *reinterpret_cast<double2*>(my_y + 2) = make_double2(py[2], py[3]);
+      *reinterpret_cast<double2*>(my_x + my_first) = make_double2(px[0], px[1]);
+      *reinterpret_cast<double2*>(my_x + (half - my_first)) = make_double2(px[2], px[3]);
+      *reinterpret_cast<double2*>(my_y + my_first) = make_double2(py[0], py[1]);
+      *reinterpret_cast<double2*>(my_y + (half - my_first)) = make_double2(py[2], py[3]);
     }
     __syncthreads();
 
@@ -154,16 +171,18 @@ __global__ void __launch_bounds__(kCsrThreads, 1) step_csr_kernel(const StepPara
       for (int e = 0; e < 4; ++e) cx[e] = cy[e] = 0.0;
       for (int k = k0; k < k1; ++k) {
         const double w = vals[k];
-        const size_t src = static_cast<size_t>(cols[k]) * pitch + 4 * cg;
+        const int col = cols[k];
+        const int first = ((col >> swz_shift) & swz_mask) * half;
+        const size_t src = piece + static_cast<size_t>(col) * pitch + 2 * cg + first, src2 = src + (half - 2 * first);
         const double2 x01 = *reinterpret_cast<const double2*>(sx + src);
-        const double2 x23 = *reinterpret_cast<const double2*>(sx + src + 2);
+        const double2 x23 = *reinterpret_cast<const double2*>(sx + src2);
         cx[0] = fma(w, x01.x, cx[0]);
         cx[1] = fma(w, x01.y, cx[1]);
         cx[2] = fma(w, x23.x, cx[2]);
         cx[3] = fma(w, x23.y, cx[3]);
         if (!dpsgd) {
           const double2 y01 = *reinterpret_cast<const double2*>(sy + src);
-          const double2 y23 = *reinterpret_cast<const double2*>(sy + src + 2);
+          const double2 y23 = *reinterpret_cast<const double2*>(sy + src2);
           cy[0] = fma(w, y01.x, cy[0]);
           cy[1] = fma(w, y01.y, cy[1]);
           cy[2] = fma(w, y23.x, cy[2]);
@@ -177,20 +196,22 @@ __global__ void __launch_bounds__(kCsrThreads, 1) step_csr_kernel(const StepPara
       }
       if (r + 1 < p.K) {
         if (owner) {  // this round's own values become the next round's "previous"
-          const double2 x01 = *reinterpret_cast<const double2*>(my_x), x23 = *reinterpret_cast<const double2*>(my_x + 2);
+          const double2 x01 = *reinterpret_cast<const double2*>(my_x + my_first);
+          const double2 x23 = *reinterpret_cast<const double2*>(my_x + (half - my_first));
           px[0] = x01.x; px[1] = x01.y; px[2] = x23.x; px[3] = x23.y;
           if (!dpsgd) {
-            const double2 y01 = *reinterpret_cast<const double2*>(my_y), y23 = *reinterpret_cast<const double2*>(my_y + 2);
+            const double2 y01 = *reinterpret_cast<const double2*>(my_y + my_first);
+            const double2 y23 = *reinterpret_cast<const double2*>(my_y + (half - my_first));
             py[0] = y01.x; py[1] = y01.y; py[2] = y23.x; py[3] = y23.y;
           }
         }
         __syncthreads();  // everybody has read round r's values
         if (owner) {
-          *reinterpret_cast<double2*>(my_x) = make_double2(cx[0], cx[1]);
-          *reinterpret_cast<double2*>(my_x + 2) = make_double2(cx[2], cx[3]);
+          *reinterpret_cast<double2*>(my_x + my_first) = make_double2(cx[0], cx[1]);
+          *reinterpret_cast<double2*>(my_x + (half - my_first)) = make_double2(cx[2], cx[3]);
           if (!dpsgd) {
-            *reinterpret_cast<double2*>(my_y) = make_double2(cy[0], cy[1]);
-            *reinterpret_cast<double2*>(my_y + 2) = make_double2(cy[2], cy[3]);
+            *reinterpret_cast<double2*>(my_y + my_first) = make_double2(cy[0], cy[1]);
+            *reinterpret_cast<double2*>(my_y + (half - my_first)) = make_double2(cy[2], cy[3]);
           }
         }
         __syncthreads();
@@ -203,7 +224,7 @@ __global__ void __launch_bounds__(kCsrThreads, 1) step_csr_kernel(const StepPara
       // lane r4 draws coordinate j + r4 for the quad's four workers; the transpose gives it its own row's four
       normal_quad(p.seed_lo, p.seed_hi, static_cast<unsigned long long>(p.coord_offset + j + r4), static_cast<uint32_t>(q),
                   p.t_noise, xi);
-      transpose_rows(xi, r4);
+      transpose_rows(xi, r4, groups);
     }
     if (active) {
       float xo[4], yo[4], go[4];
@@ -247,19 +268,26 @@ __global__ void __launch_bounds__(kCsrThreads, 1) step_csr_kernel(const StepPara
 
 }  // namespace
 
-// Chooses the slab width: the widest power of two (4 .. 64 coordinates) for which every (worker quad, four
+// Chooses the slab width: the widest power of two (4 .. 32 coordinates) for which every (worker quad, four
 // coordinates) item has a thread of its own and the slabs fit; the CSR arrays join them in shared memory if there
 // is room.  p.log2S < 0 afterwards means the tables stay in global memory.
 int plan_step_csr(StepParams& p, int smem_optin_bytes) {
   const int quads = (p.n + 3) / 4;
   int best = 0;
-  for (int S = 64; S >= 4; S >>= 1) {
+  for (int S = kCsrMaxS; S >= 4; S >>= 1) {
     if (quads * 4 * (S / 4) > kCsrThreads) continue;
     if (csr_smem_bytes(p.n, p.nnz, S, false) > static_cast<size_t>(smem_optin_bytes)) continue;
     best = S;
     break;
   }
   if (best == 0) return DETAG_ERR_UNSUPPORTED;
+  // small graphs: as many pieces of that width as threads and shared memory allow (at most 8)
+  int pieces = 1;
+  while (pieces < 8 && quads * 4 * (best / 4) * (pieces * 2) <= kCsrThreads &&
+         csr_smem_bytes(p.n, p.nnz, best * pieces * 2, true) <= static_cast<size_t>(smem_optin_bytes))
+    pieces *= 2;
+  p.csr_sub = pieces;
+  best *= pieces;
   p.S = best;
   p.log2S = csr_smem_bytes(p.n, p.nnz, best, true) <= static_cast<size_t>(smem_optin_bytes) ? 1 : -1;
   p.num_slabs = (p.d + best - 1) / best;
@@ -269,7 +297,9 @@ int plan_step_csr(StepParams& p, int smem_optin_bytes) {
 int launch_step_csr(const StepParams& p, int sm_count, cudaStream_t stream) {
   const bool tables = p.log2S > 0;
   const size_t smem = csr_smem_bytes(p.n, p.nnz, p.S, tables);
-  auto kernel = tables ? step_csr_kernel<true> : step_csr_kernel<false>;
+  const bool swap = p.S / p.csr_sub < kCsrMaxS;
+  auto kernel = tables ? (swap ? step_csr_kernel<true, true> : step_csr_kernel<true, false>)
+                       : (swap ? step_csr_kernel<false, true> : step_csr_kernel<false, false>);
   const int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), static_cast<int>(smem));
   if (rc != 0) return rc;
   const long long grid = p.num_slabs < static_cast<long long>(sm_count) ? p.num_slabs : static_cast<long long>(sm_count);
