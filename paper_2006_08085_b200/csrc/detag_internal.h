@@ -27,6 +27,7 @@ struct StepParams {
   int S;           // slab width in coordinates (power of two)
   int log2S;
   int csr_sub;     // generic rounds kernel: independent pieces the slab is cut into
+  int csr_threads; // generic rounds kernel: threads per block (1024, or 512 with two blocks per SM)
   long long d;
   long long ld;
   long long num_slabs;
