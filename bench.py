@@ -51,6 +51,7 @@ MEASURED_TRAFFIC = {
     ("torus", "torus8"): ("427a2bff49b63d9c", 31.27),  # cfg3 shape at d = 1 M: 1.2803 + 0.7208 GB / 64 M wc
     ("ring", "band"): ("60c16ee651aa8e4f", 31.12),     # cfg4 shape at d = 200 k: 1.0280 + 0.5652 GB / 51.2 M wc
     ("wide", "dense"): ("77d5b7be943b4c42", 30.83),    # 100-worker random graph at d = 400 k: 0.8011 + 0.4321 GB / 40 M wc
+    ("csr", "rounds"): ("bcc2ab2f791da0eb", 31.17),    # the same graph through the rounds kernel: 0.8088 + 0.4381 GB / 40 M wc
 }
 
 # Float64 multiply-adds per worker-coordinate on the FP64 pipe (both contractions, padded shapes) and that
