@@ -274,7 +274,19 @@ int resolve_variant(const detag_state* s) {
   if (step_mode(s) != detag::kModeDetag) return (s->n <= 32 && dense_ok(s)) ? DETAG_VARIANT_DENSE : DETAG_VARIANT_CSR;
   if (s->n > 32 && ring) return DETAG_VARIANT_RING;
   if (s->n > 32 && torus_ok(s)) return DETAG_VARIANT_TORUS;
-  if (dense_ok(s)) return DETAG_VARIANT_DENSE;
+  if (dense_ok(s)) {
+    if (s->n > detag::kMaxDenseWorkers) {
+      // Register-resident polynomial against the sparse rounds, both measured at d = 2 M (ms): the dense kernel is
+      // bound by one warp scheduler's share of the MMAs - blocks / 4 strips (the next multiple of four when one
+      // scheduler is a block short) of n / 4 k-steps - the rounds kernel by a per-worker part and K * nnz
+      // shared-memory gathers.  The rounds win at one or two rounds on graphs of degree four.
+      const int blocks = (s->n + 7) / 8, blocks_eff = blocks % 4 == 3 ? blocks + 1 : blocks;
+      const double dense_ms = 0.0412 * blocks_eff * blocks / 2.0;
+      const double rounds_ms = 0.024 * s->n + 0.00155 * s->K * static_cast<double>(s->col_idx.size());
+      if (rounds_ms < dense_ms) return DETAG_VARIANT_CSR;
+    }
+    return DETAG_VARIANT_DENSE;
+  }
   return DETAG_VARIANT_CSR;
 }
 

@@ -327,8 +327,10 @@ def test_dense_polynomial_held_in_registers(n, d, K, kind):
         picked = B.detag_get_variant(st)
     finally:
         B.detag_destroy(st)
-    if kind in ("regular4", "path"):
-        assert picked == B.DETAG_VARIANT_DENSE  # no structure: the dense polynomial is the default
+    if kind == "regular4":
+        assert picked == B.DETAG_VARIANT_DENSE  # no structure, several rounds: the dense polynomial
+    if kind == "path":
+        assert picked == B.DETAG_VARIANT_CSR    # three rounds over two neighbours: the sparse rounds are cheaper
     a, c = _random_objective(rng, n, d, scale=0.1)
     x0 = rng.standard_normal((n, d)).astype(np.float32)
     variants = [B.DETAG_VARIANT_DENSE]
